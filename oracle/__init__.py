@@ -1,0 +1,231 @@
+"""ctypes loader for the CPU oracle (oracle/disc_oracle.cpp).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never
+import this package, and this package never imports them.
+
+The shared object is compiled on first use with g++ (a few seconds).
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "disc_oracle.cpp")
+_LIB = os.path.join(_HERE, "libdisc_oracle.so")
+
+ERR_ARG, ERR_EMPTY, ERR_TOKEN, ERR_PREFIX, ERR_UNSUPPORTED = -1, -2, -3, -4, -7
+F32, BF16 = 0, 1
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle if the shared object is missing or older than the source."""
+    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    if force or stale:
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.run(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", "-o", tmp, _SRC],
+                       check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        L = C.CDLL(build())
+        vp, i32, i64, u32, u64 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64
+        L.oracle_build.argtypes = [vp, vp, i64, i32, C.POINTER(vp)]
+        L.oracle_build.restype = C.c_int
+        L.oracle_free.argtypes = [vp]
+        L.oracle_free.restype = None
+        L.oracle_info.argtypes = [vp, vp]
+        L.oracle_info.restype = None
+        L.oracle_rows.argtypes = [vp, vp, vp]
+        L.oracle_rows.restype = None
+        L.oracle_mask.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp]
+        L.oracle_mask.restype = None
+        L.oracle_step.argtypes = [vp, vp, C.c_int, i64, i64, C.c_float, u64, u32, vp,
+                                  vp, i32, vp, vp, vp,
+                                  vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
+        L.oracle_step.restype = None
+        L.oracle_resample.argtypes = [vp, i32, i32, u64, vp, vp, vp, vp, vp, vp]
+        L.oracle_resample.restype = None
+        L.oracle_accept.argtypes = [vp, i32, i32, u64, vp, vp]
+        L.oracle_accept.restype = None
+        L.oracle_decode_markov.argtypes = [vp, vp, vp, i32, i32, C.c_float, u64, i64,
+                                           vp, vp, vp, vp, vp, vp, C.c_int]
+        L.oracle_decode_markov.restype = C.c_int
+        L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
+        L.oracle_philox4x32_10.restype = None
+        L.oracle_gumbel_uniform.argtypes = [u64, u32, u32, u32]
+        L.oracle_gumbel_uniform.restype = C.c_double
+        L.oracle_resample_uniform.argtypes = [u64, u32]
+        L.oracle_resample_uniform.restype = C.c_double
+        L.oracle_accept_uniform.argtypes = [u64, u32, u32]
+        L.oracle_accept_uniform.restype = C.c_double
+        _lib = L
+    return _lib
+
+
+def _p(a):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _c(a, dtype):
+    return np.ascontiguousarray(a, dtype=dtype)
+
+
+class OracleError(RuntimeError):
+    def __init__(self, code):
+        super().__init__(f"oracle_build failed with code {code}")
+        self.code = code
+
+
+class OracleSet:
+    """The constraint set as an explicit prefix tree."""
+
+    def __init__(self, tokens, row_offsets, vocab_size):
+        tokens = _c(tokens, np.int32)
+        row_offsets = _c(row_offsets, np.int64)
+        h = C.c_void_p()
+        rc = lib().oracle_build(_p(tokens), _p(row_offsets), row_offsets.shape[0] - 1,
+                                int(vocab_size), C.byref(h))
+        if rc != 0:
+            raise OracleError(rc)
+        self._h = h
+        info = np.zeros(4, dtype=np.int64)
+        lib().oracle_info(self._h, _p(info))
+        self.N, self.E, self.l_max, self.n_nodes = (int(x) for x in info)
+        self.V = int(vocab_size)
+        self.W = (self.V + 31) // 32
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().oracle_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    def rows(self):
+        """Sorted, de-duplicated table: (tokens int32[E], row_offsets int64[N+1])."""
+        tok = np.empty(self.E, dtype=np.int32)
+        off = np.empty(self.N + 1, dtype=np.int64)
+        lib().oracle_rows(self._h, _p(tok), _p(off))
+        return tok, off
+
+    def mask(self, prefix, prefix_len):
+        prefix = _c(prefix, np.int32)
+        if prefix.ndim == 1:
+            prefix = prefix.reshape(1, -1)
+        prefix_len = _c(prefix_len, np.int32).reshape(-1)
+        n = prefix_len.shape[0]
+        ld = prefix.shape[1] if prefix.shape[1] > 0 else 1
+        if prefix.shape[1] == 0:
+            prefix = np.zeros((n, 1), dtype=np.int32)
+        mask = np.empty((n, self.W), dtype=np.uint32)
+        lo = np.empty(n, dtype=np.int32)
+        hi = np.empty(n, dtype=np.int32)
+        status = np.empty(n, dtype=np.uint8)
+        lib().oracle_mask(self._h, _p(prefix), ld, _p(prefix_len), n, _p(mask), _p(lo), _p(hi), _p(status))
+        return mask, lo, hi, status
+
+    def step(self, logits, dtype, prefix, depth, done=None, *, inv_temperature=1.0, seed=0, step=0,
+             row_ids=None, alt_token=None, n_threads=1):
+        """One decoding step.  logits: [n, ld] float32 array, or uint16 array holding bf16 bits."""
+        depth = _c(depth, np.int32).reshape(-1)
+        n = depth.shape[0]
+        logits = np.ascontiguousarray(logits)
+        assert logits.ndim == 2 and logits.shape[0] == n and logits.shape[1] >= self.V
+        assert logits.dtype == (np.float32 if dtype == F32 else np.uint16)
+        prefix = _c(prefix, np.int32)
+        if prefix.ndim == 1:
+            prefix = prefix.reshape(n, -1)
+        if prefix.shape[1] == 0:
+            prefix = np.zeros((n, 1), dtype=np.int32)
+        done = None if done is None else _c(done, np.uint8)
+        row_ids = None if row_ids is None else _c(row_ids, np.int64)
+        alt_token = None if alt_token is None else _c(alt_token, np.int32)
+        o = {
+            "token": np.empty(n, np.int32), "lo": np.empty(n, np.int32), "hi": np.empty(n, np.int32),
+            "done": np.empty(n, np.uint8), "log_mass": np.empty(n), "lse_all": np.empty(n),
+            "lse_ok": np.empty(n), "logq": np.empty(n), "logp": np.empty(n), "best": np.empty(n),
+            "second": np.empty(n), "alt": np.empty(n), "n_children": np.empty(n, np.int32),
+            "status": np.empty(n, np.uint8),
+        }
+        lib().oracle_step(self._h, _p(logits), int(dtype), logits.shape[1], n, float(inv_temperature),
+                          int(seed), int(step), _p(row_ids), _p(prefix), prefix.shape[1], _p(depth),
+                          _p(done), _p(alt_token),
+                          _p(o["token"]), _p(o["lo"]), _p(o["hi"]), _p(o["done"]), _p(o["log_mass"]),
+                          _p(o["lse_all"]), _p(o["lse_ok"]), _p(o["logq"]), _p(o["logp"]),
+                          _p(o["best"]), _p(o["second"]), _p(o["alt"]), _p(o["n_children"]),
+                          _p(o["status"]), int(n_threads))
+        return o
+
+    def decode_markov(self, Z, ctx, K, *, inv_temperature=1.0, seed=0, query_base=0, n_threads=1):
+        """Free-running SampleCandidate x (B*K) + K-way draw under a Markov LM table Z[V, V]."""
+        Z = _c(Z, np.float32)
+        assert Z.shape == (Z.shape[0], self.V)
+        ctx = _c(ctx, np.int32)
+        B = ctx.shape[0]
+        L = self.l_max
+        o = {
+            "seq": np.empty((B, K, L), np.int32), "len": np.empty((B, K), np.int32),
+            "logw": np.empty((B, K)), "logw32": np.empty((B, K), np.float32),
+            "idx": np.empty(B, np.int32), "logz": np.empty(B),
+        }
+        rc = lib().oracle_decode_markov(self._h, _p(Z), _p(ctx), B, K, float(inv_temperature), int(seed),
+                                        int(query_base), _p(o["seq"]), _p(o["len"]), _p(o["logw"]),
+                                        _p(o["logw32"]), _p(o["idx"]), _p(o["logz"]), int(n_threads))
+        assert rc == 0
+        return o
+
+
+def resample(logw, seed=0, query_ids=None):
+    logw = _c(logw, np.float32)
+    B, K = logw.shape
+    query_ids = None if query_ids is None else _c(query_ids, np.int64)
+    o = {"idx": np.empty(B, np.int32), "logz": np.empty(B), "u": np.empty(B), "gap": np.empty(B),
+         "status": np.empty(B, np.uint8)}
+    lib().oracle_resample(_p(logw), B, K, int(seed), _p(query_ids), _p(o["idx"]), _p(o["logz"]),
+                          _p(o["u"]), _p(o["gap"]), _p(o["status"]))
+    return o
+
+
+def accept(logw, seed=0, query_ids=None):
+    logw = _c(logw, np.float32)
+    B, K = logw.shape
+    query_ids = None if query_ids is None else _c(query_ids, np.int64)
+    out = np.empty(B, np.int32)
+    lib().oracle_accept(_p(logw), B, K, int(seed), _p(query_ids), _p(out))
+    return out
+
+
+def philox4x32_10(ctr, key):
+    ctr = _c(ctr, np.uint32)
+    key = _c(key, np.uint32)
+    out = np.empty(4, np.uint32)
+    lib().oracle_philox4x32_10(_p(ctr), _p(key), _p(out))
+    return out
+
+
+def gumbel_uniform(seed, step, row, v):
+    return lib().oracle_gumbel_uniform(int(seed), int(step), int(row), int(v))
+
+
+def resample_uniform(seed, query):
+    return lib().oracle_resample_uniform(int(seed), int(query))
+
+
+def accept_uniform(seed, query, k):
+    return lib().oracle_accept_uniform(int(seed), int(query), int(k))

@@ -1,0 +1,195 @@
+"""Pins for the oracle's table build, valid-set masks and member ranges.
+
+The oracle builds a prefix tree by insertion; these tests compare it with what
+the definitions fix, computed a different way: Python's built-in sort of tuples
+(lexicographic, shorter-first), a scan over every member for the valid set
+(Section 2.1), and the lower-bound characterisation of Section 3.2
+("t_m is valid iff V_m is a prefix of the row the binary search lands on").
+"""
+import bisect
+import itertools
+import os
+
+import numpy as np
+import pytest
+
+import oracle
+from workloads import CONFIGS, make_set, scaled
+
+
+def _csr(rows):
+    tok = np.array([t for r in rows for t in r], dtype=np.int32)
+    off = np.zeros(len(rows) + 1, dtype=np.int64)
+    off[1:] = np.cumsum([len(r) for r in rows])
+    return tok, off
+
+
+def _rows_of(tok, off):
+    return [tuple(int(x) for x in tok[off[i]:off[i + 1]]) for i in range(len(off) - 1)]
+
+
+def _is_prefix(a, s):
+    return len(a) <= len(s) and tuple(s[:len(a)]) == tuple(a)
+
+
+def _brute_mask(members, a, V):
+    """A_{a,S} by scanning every member, plus the member range of prefix a."""
+    allowed = {v for v in range(V) if any(_is_prefix(tuple(a) + (v,), s) for s in members)}
+    n_with = sum(_is_prefix(a, s) for s in members)
+    if n_with == 0:
+        return None
+    lo = sum(1 for s in members if s < tuple(a))
+    return allowed, lo, lo + n_with
+
+
+def _bits(mask_row, V):
+    return {v for v in range(V) if (int(mask_row[v >> 5]) >> (v & 31)) & 1}
+
+
+def _random_prefix_free_set(rng, V, L_max, n, eos):
+    rows = set()
+    for _ in range(n):
+        if eos:
+            ell = int(rng.integers(1, L_max))
+            rows.add(tuple(int(x) for x in rng.integers(0, V - 1, size=ell)) + (V - 1,))
+        else:
+            rows.add(tuple(int(x) for x in rng.integers(0, V, size=L_max)))
+    return list(rows)
+
+
+def test_sorted_table_equals_library_sort_tiny_config():
+    w = CONFIGS["tiny"]
+    tok, off = make_set(w)
+    S = oracle.OracleSet(tok, off, w.V)
+    expect = sorted(set(_rows_of(tok, off)))
+    got = _rows_of(*S.rows())
+    assert got == expect
+    assert S.N == len(expect) == 256 and S.l_max == 3 and S.E == 768
+
+
+@pytest.mark.parametrize("name,n", [("genret", 5000), ("llm", 20000), ("large", 20000)])
+def test_sorted_table_equals_library_sort_scaled(name, n):
+    w = scaled(name, n_draws=n)
+    tok, off = make_set(w)
+    S = oracle.OracleSet(tok, off, w.V)
+    expect = sorted(set(_rows_of(tok, off)))
+    assert _rows_of(*S.rows()) == expect
+    assert S.N == len(expect)
+    assert S.l_max == max(len(r) for r in expect)
+
+
+def test_duplicates_collapse_and_input_order_is_irrelevant():
+    rows = [(3, 1), (0, 2), (3, 1), (0, 1), (3, 0)]
+    a = oracle.OracleSet(*_csr(rows), 4)
+    b = oracle.OracleSet(*_csr(rows[::-1]), 4)
+    assert _rows_of(*a.rows()) == _rows_of(*b.rows()) == [(0, 1), (0, 2), (3, 0), (3, 1)]
+
+
+@pytest.mark.parametrize("rows,V,code", [
+    ([(1, 2), ()], 4, oracle.ERR_EMPTY),
+    ([(1, 2), (1, 4)], 4, oracle.ERR_TOKEN),
+    ([(1, 2), (-1, 0)], 4, oracle.ERR_TOKEN),
+    ([(1, 2), (1, 2, 3)], 4, oracle.ERR_PREFIX),
+    ([(1, 2, 3), (1, 2)], 4, oracle.ERR_PREFIX),
+    ([], 4, oracle.ERR_EMPTY),
+])
+def test_build_rejects(rows, V, code):
+    with pytest.raises(oracle.OracleError) as e:
+        oracle.OracleSet(*_csr(rows), V)
+    assert e.value.code == code
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("eos", [False, True])
+def test_mask_and_range_brute_force_all_prefixes(seed, eos):
+    rng = np.random.default_rng(1000 + seed)
+    V = int(rng.integers(2, 9))
+    L = int(rng.integers(2, 5))
+    members = _random_prefix_free_set(rng, V, L, int(rng.integers(1, 40)), eos)
+    S = oracle.OracleSet(*_csr(members), V)
+    members = sorted(members)
+    # every sequence of length 0..L over the vocabulary, member prefix or not
+    for ell in range(L + 1):
+        for a in itertools.product(range(V), repeat=ell):
+            pref = np.zeros((1, max(L, 1)), np.int32)
+            pref[0, :ell] = a
+            mask, lo, hi, status = S.mask(pref, [ell])
+            bm = _brute_mask(members, a, V)
+            if bm is None:
+                assert status[0] == 1 and lo[0] == -1 and hi[0] == -1 and not mask.any()
+                continue
+            allowed, blo, bhi = bm
+            assert status[0] == 0
+            assert _bits(mask[0], V) == allowed
+            assert (int(lo[0]), int(hi[0])) == (blo, bhi)
+            # a complete member has an empty valid set and a range of one row
+            if tuple(a) in members:
+                assert not allowed and bhi - blo == 1
+            # partition invariant: children's ranges tile the parent's range
+            tot, cursor = 0, blo
+            for v in sorted(allowed):
+                p2 = pref.copy()
+                p2[0, ell] = v if ell < pref.shape[1] else 0
+                if ell >= pref.shape[1]:
+                    continue
+                _, clo, chi, cst = S.mask(p2, [ell + 1])
+                assert cst[0] == 0 and clo[0] == cursor
+                cursor = int(chi[0])
+                tot += int(chi[0] - clo[0])
+            if allowed:
+                assert tot == bhi - blo and cursor == bhi
+
+
+@pytest.mark.parametrize("name,n", [("tiny", 256), ("llm", 3000), ("large", 3000)])
+def test_mask_matches_lower_bound_characterisation(name, n):
+    """Section 3.2: v is valid after prefix a iff a+[v] is a prefix of the first row >= a+[v]."""
+    w = scaled(name, n_draws=n)
+    tok, off = make_set(w)
+    S = oracle.OracleSet(tok, off, w.V)
+    table = _rows_of(*S.rows())
+    rng = np.random.default_rng(7)
+    for _ in range(25):
+        r = table[int(rng.integers(0, len(table)))]
+        ell = int(rng.integers(0, len(r)))
+        a = r[:ell]
+        pref = np.zeros((1, S.l_max), np.int32)
+        pref[0, :ell] = a
+        mask, lo, hi, status = S.mask(pref, [ell])
+        assert status[0] == 0
+        got = _bits(mask[0], w.V)
+        # check every token of a small vocabulary, a sample (plus all set bits) of a large one
+        cand = range(w.V) if w.V <= 64 else set(rng.integers(0, w.V, 300).tolist()) | got
+        for v in cand:
+            key = a + (v,)
+            i = bisect.bisect_left(table, key)
+            valid = i < len(table) and _is_prefix(key, table[i])
+            assert (v in got) == valid
+        assert int(lo[0]) == bisect.bisect_left(table, a)
+        assert int(hi[0]) - int(lo[0]) == sum(_is_prefix(a, s) for s in table[int(lo[0]):int(hi[0]) + 1])
+
+
+def test_full_set_gives_all_ones_and_single_member_gives_one_bit():
+    V, L = 5, 3
+    full = list(itertools.product(range(V), repeat=L))
+    S = oracle.OracleSet(*_csr(full), V)
+    for ell in range(L):
+        for a in itertools.product(range(V), repeat=ell):
+            pref = np.zeros((1, L), np.int32)
+            pref[0, :ell] = a
+            mask, lo, hi, st = S.mask(pref, [ell])
+            assert _bits(mask[0], V) == set(range(V))
+            assert int(hi[0] - lo[0]) == V ** (L - ell)
+    one = oracle.OracleSet(*_csr([(4, 0, 2)]), V)
+    for ell, want in [(0, {4}), (1, {0}), (2, {2}), (3, set())]:
+        pref = np.array([[4, 0, 2]], np.int32)
+        mask, lo, hi, st = one.mask(pref, [ell])
+        assert _bits(mask[0], V) == want and (int(lo[0]), int(hi[0])) == (0, 1)
+
+
+def test_bits_beyond_vocabulary_are_zero():
+    V = 37
+    rows = [(v, 0) for v in range(V)]
+    S = oracle.OracleSet(*_csr(rows), V)
+    mask, *_ = S.mask(np.zeros((1, 2), np.int32), [0])
+    assert mask.shape == (1, 2)
+    assert int(mask[0, 0]) == 0xFFFFFFFF and int(mask[0, 1]) == (1 << 5) - 1
