@@ -1,0 +1,469 @@
+#!/usr/bin/env python
+"""Benchmark of the DISC + PPV hot path on the "large" workload (V = 128,256).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload large]
+
+One "step" is one whole decode of the workload's B*K candidates: disc_state_init, one disc_step per
+token position (l_max launches; finished rows cost nothing), disc_resample.  The stand-in language
+model is outside the timed region: its logits for every position are produced once by a recording
+decode and kept resident in HBM (1.05 GB per position at the large workload, so every launch
+streams far more than the L2 holds); the timed decodes replay them with the same seed and so
+reproduce the same tokens.  Prints ONE JSON line (rank 0).
+
+--impl reference times the CPU oracle (oracle/) as it stands on the host cores, on a bounded sample
+of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "disc_decode_tokens_per_s"
+UNIT = "tokens/s"
+# DRAM bytes per disc_step launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum),
+# as a ratio to the algorithmic bytes of the captured launch; None until a capture exists.
+# Source: profiles/disc_step_large.md
+NCU_TRAFFIC_RATIO = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="large", choices=["tiny", "genret", "llm", "large"])
+    ap.add_argument("--draws", type=int, default=0, help="override the number of members drawn (debugging)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-sample-rows", type=int, default=256)
+    return ap.parse_args()
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return float(d["hbm_gbs"]), "measured"
+    return 6650.0, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons through NVML (read-only) while the timed region runs."""
+
+    def __init__(self, index: int):
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop = threading.Event()
+        self._t = None
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = int(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception:
+            self.nv = None
+
+    def _run(self):
+        nv = self.nv
+        names = {"hw_slowdown": nv.nvmlClocksThrottleReasonHwSlowdown,
+                 "hw_thermal_slowdown": nv.nvmlClocksThrottleReasonHwThermalSlowdown,
+                 "sw_thermal_slowdown": nv.nvmlClocksThrottleReasonSwThermalSlowdown,
+                 "sw_power_cap": nv.nvmlClocksThrottleReasonSwPowerCap}
+        while not self._stop.is_set():
+            try:
+                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                r = int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h))
+                for k, bit in names.items():
+                    if r & bit:
+                        self.reasons.add(k)
+            except Exception:
+                pass
+            self._stop.wait(0.02)
+
+    def start(self):
+        if self.nv is not None:
+            self._t = threading.Thread(target=self._run, daemon=True)
+            self._t.start()
+
+    def stop(self):
+        self._stop.set()
+        if self._t is not None:
+            self._t.join()
+        med = int(np.median(self.samples)) if self.samples else None
+        return {"sm_mhz": med, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons),
+                "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank: int) -> int:
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def popcount_rows(mask):
+    """Set bits per row of an int32 [n, W] device tensor (bookkeeping for the byte count only)."""
+    import torch
+    table = torch.tensor([bin(i).count("1") for i in range(256)], dtype=torch.int32, device=mask.device)
+    return table[mask.contiguous().view(torch.uint8).to(torch.int64)].view(mask.shape[0], -1).sum(1)
+
+
+def logits_to_numpy(t):
+    """Logits tensor -> (numpy array of the same bytes, oracle dtype code)."""
+    import torch
+    if t.dtype == torch.float32:
+        return t.detach().cpu().numpy(), 0
+    return t.detach().view(torch.int16).cpu().numpy().view(np.uint16), 1
+
+
+def workload(args):
+    from workloads import CONFIGS, scaled
+    w = CONFIGS[args.workload]
+    if args.draws:
+        w = scaled(args.workload, n_draws=args.draws)
+    return w
+
+
+def describe(w, N=None):
+    s = (f"{w.name}: V={w.V}, {w.n_draws} members drawn (len {w.len_min}-{w.len_max}"
+         f"{', EOS-closed' if w.eos else ''}, {w.token_dist} tokens), B={w.B}, K={w.K}, {w.logits} logits, "
+         f"stand-in LM d={w.d}")
+    if N is not None:
+        s += f", |S|={N} after de-duplication"
+    return s
+
+
+# ------------------------------------------------------------------------------------------ ours
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    import paper_2504_09135_b200 as disc
+    from workloads import make_contexts, make_lm_weights, make_set
+    from workloads.standin_lm import StandInLM
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    w = workload(args)
+    t_setup = time.time()
+
+    # the constraint set is replicated on every GPU; each rank decodes its own queries
+    tok, off = make_set(w)
+    G = disc.disc_build_set(tok, off, w.V)
+    lm = StandInLM(*make_lm_weights(w), w.logits, dev)
+    ctx = torch.as_tensor(make_contexts(w, salt=rank), device=dev)
+    dec = disc.DiscDecoder(G, w.B, w.K, dev)
+    seed = 250409135 + rank
+    L = G.l_max
+    esize = 4 if w.logits == "f32" else 2
+
+    # ---- recording decode: keep every position's logits; count live rows and valid-set sizes
+    logits_steps, alive, children = [], [], []
+    dec.reset()
+    prev = ctx.to(torch.int64).repeat_interleave(w.K)
+    mask_buf = torch.empty((dec.R, G.W), dtype=torch.int32, device=dev)
+    probe = disc.StepOutputs.empty(dec.R, dev, mask_words=0)
+    probe.mask = mask_buf
+    for t in range(L):
+        logits = lm.logits(prev)
+        live = (dec.state.done == 0)
+        alive.append(int(live.sum().item()))
+        st_copy = dec.state.clone()
+        disc.disc_step(G, logits, st_copy, seed=seed, step=t, out=probe)       # mask only, state copy
+        c = popcount_rows(mask_buf)
+        children.append(int(c[0].item()) if t == 0 else int((c * live).sum().item()))
+        o = dec.step(logits, t, seed=seed)
+        prev = torch.where(o.token >= 0, o.token.to(torch.int64), prev)
+        logits_steps.append(logits)
+    first = dec.finish(seed=seed)
+    first_tokens = first["tokens"].clone()
+    first_logw = dec.state.logw.clone()
+    torch.cuda.synchronize()
+    assert bool(dec.state.done.all()), "decode did not finish within l_max steps"
+    del mask_buf, probe
+    tokens_per_decode = int(sum(alive))
+    launches = [t for t in range(L) if alive[t] > 0]
+    alg_bytes = [alive[t] * (w.V * esize + 46) + 4 * children[t] for t in range(L)]
+
+    # ---- stand-in LM projection, timed separately (outside the hot path)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    scratch_logits = torch.empty_like(logits_steps[0])
+    lm.logits(prev, out=scratch_logits) if lm.b is None else lm.logits(prev)
+    torch.cuda.synchronize()
+    e0.record()
+    for _ in range(3):
+        lm.logits(prev, out=scratch_logits) if lm.b is None else lm.logits(prev)
+    e1.record()
+    torch.cuda.synchronize()
+    lm_ms = e0.elapsed_time(e1) / 3
+    del scratch_logits
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K whole decodes over the resident logits
+    for _ in range(max(args.warmup, 3)):
+        dec.replay(logits_steps, seed=seed)
+    barrier()
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    sampler.start()
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(L)]
+          for _ in range(args.steps)]
+    t0, t1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    t0.record()
+    for k in range(args.steps):
+        dec.reset()
+        for t in range(L):
+            ev[k][t][0].record()
+            dec.step(logits_steps[t], t, seed=seed)
+            ev[k][t][1].record()
+        dec.finish(seed=seed)
+    t1.record()
+    barrier()
+    clocks = sampler.stop()
+    total_ms = t0.elapsed_time(t1)
+    same_tokens = bool(torch.equal(dec.res["tokens"], first_tokens)) and bool(torch.equal(dec.state.logw, first_logw))
+    step_ms = np.array([[ev[k][t][0].elapsed_time(ev[k][t][1]) for t in range(L)] for k in range(args.steps)])
+    if world > 1:
+        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+        total_ms = float(tt.item())
+    value = world * args.steps * tokens_per_decode / (total_ms * 1e-3)
+    gpu_launches = args.steps * (1 + L + 1)      # disc_state_init + L x disc_step + disc_resample
+
+    # roofline of the dominant kernel (disc_step): algorithmic bytes / device time, launches with live rows
+    kern_ms = float(step_ms[:, launches].sum())
+    kern_bytes = float(sum(alg_bytes[t] for t in launches)) * args.steps
+    achieved = kern_bytes / (kern_ms * 1e-3) / 1e9
+    peak, peak_kind = measured_peaks()
+    per_step = [{"step": t, "live_rows": alive[t], "ms": round(float(step_ms[:, t].mean()), 4),
+                 "gbs": round(alg_bytes[t] / (float(step_ms[:, t].mean()) * 1e-3) / 1e9, 1)} for t in launches]
+    roofline = {"bound": "hbm", "kernel": "disc_step_kernel", "achieved": round(achieved, 1), "peak": peak,
+                "unit": "GB/s", "frac": round(achieved / peak, 4), "peak_kind": f"of {peak_kind}",
+                "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
+                "alg_bytes_per_launch": int(kern_bytes / args.steps / len(launches)),
+                "avg_launch_ms": round(kern_ms / args.steps / len(launches), 4),
+                "traffic": (None if NCU_TRAFFIC_RATIO is None
+                            else int(NCU_TRAFFIC_RATIO * kern_bytes / args.steps / len(launches))),
+                "per_step": per_step}
+
+    # ---- end to end: logits start in pinned host memory, result read back to the host
+    e2e = None
+    if not args.no_e2e:
+        host = [torch.empty(l.shape, dtype=l.dtype, pin_memory=True) for l in logits_steps]
+        for h, l in zip(host, logits_steps):
+            h.copy_(l)
+        staging = torch.empty_like(logits_steps[0])
+        torch.cuda.synchronize()
+        dec.replay_from_host(host, staging, seed=seed)
+        barrier()
+        n_e2e = max(1, min(args.steps, 3))
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        wall0 = time.perf_counter()
+        a.record()
+        for _ in range(n_e2e):
+            r = dec.replay_from_host(host, staging, seed=seed)
+        b.record()
+        barrier()
+        wall = time.perf_counter() - wall0
+        e2e_ms = max(a.elapsed_time(b), wall * 1e3)
+        if world > 1:
+            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
+            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+            e2e_ms = float(tt.item())
+        assert torch.equal(r["tokens"], first_tokens.cpu())
+        h2d = int(sum(h.numel() * h.element_size() for h in host))
+        d2h = int(sum(v.numel() * v.element_size() for v in r.values()))
+        e2e = {"value": round(world * n_e2e * tokens_per_decode / (e2e_ms * 1e-3), 1), "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "decodes": n_e2e}
+        del host, staging
+
+    # ---- mask-only stress (secondary figure): 65,536 prefixes of the same table
+    mask_stress = None
+    if rank == 0 and w.name == "large":
+        from workloads import CONFIGS, make_prefixes
+        mw = CONFIGS["mask"]
+        prefix, plen = make_prefixes(mw, tok, off)
+        pre_d, len_d = torch.as_tensor(prefix, device=dev), torch.as_tensor(plen, device=dev)
+        out = disc.disc_mask(G, pre_d, len_d)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        for _ in range(3):
+            disc.disc_mask(G, pre_d, len_d, out=out)
+        a.record()
+        for _ in range(10):
+            disc.disc_mask(G, pre_d, len_d, out=out)
+        b.record()
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / 10
+        nbytes = prefix.shape[0] * G.W * 4
+        mask_stress = {"prefixes": int(prefix.shape[0]), "ms": round(ms, 4),
+                       "prefixes_per_s": round(prefix.shape[0] / (ms * 1e-3), 1),
+                       "mask_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
+                       "frac": round(nbytes / (ms * 1e-3) / 1e9 / peak, 4)}
+        del out
+
+    # ---- CPU baseline: the oracle as it stands, on a bounded sample, rank 0 at N = 1 only
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        seq = dec.seq.cpu().numpy()
+        cpu = cpu_baseline(w, tok, off, [l[:args.cpu_sample_rows] for l in logits_steps], seq[:args.cpu_sample_rows],
+                           seed)
+
+    if rank == 0:
+        line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+                "warmup": max(args.warmup, 3), "ms_per_step": round(total_ms / args.steps, 4),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic", "impl": "ours",
+                "config": {"workload": describe(w, G.N), "tokens_per_decode": tokens_per_decode,
+                           "positions": L, "logits_bytes_per_decode": int(sum(alive) * w.V * esize),
+                           "l2": "inputs larger than L2: every launch streams its own logits buffer "
+                                 f"({dec.R * w.V * esize / 1e6:.0f} MB), no flush needed",
+                           "parallelism": f"replicated set, queries sharded over {world} GPU(s), no collective"},
+                "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
+                "clocks": clocks, "deterministic_replay": same_tokens,
+                "lm_projection_ms_per_position": round(lm_ms, 3), "mask_stress": mask_stress,
+                "set": {"members": G.N, "entries": G.E, "index_nodes": G.n_nodes,
+                        "device_mb": round(G.device_bytes / 1e6, 1), "build_s": round(G.build_seconds, 3)},
+                "setup_s": round(time.time() - t_setup, 1)}
+        print(json.dumps(line))
+    G.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+# ----------------------------------------------------------------------------- oracle on the host
+def cpu_baseline(w, tok, off, logits_rows, seq, seed):
+    """Times oracle.step on the sampled rows over every position (teacher-forced on the GPU's own
+    tokens, so each call does the work of the corresponding disc_step rows)."""
+    import oracle
+    cores = os.cpu_count() or 1
+    t0 = time.time()
+    S = oracle.OracleSet(tok, off, w.V)
+    build_s = time.time() - t0
+    n = seq.shape[0]
+    lens = (seq >= 0).sum(1)
+    host = [logits_to_numpy(l) for l in logits_rows]
+
+    def run(rows, n_threads):
+        toks, secs = 0, 0.0
+        for t, (hl, dt) in enumerate(host):
+            done = (lens[:rows] <= t).astype(np.uint8)
+            if done.all():
+                break
+            a = time.perf_counter()
+            S.step(hl[:rows], dt, seq[:rows], np.full(rows, t, np.int32), done, seed=seed, step=t, n_threads=n_threads)
+            secs += time.perf_counter() - a
+            toks += int((done == 0).sum())
+        return toks, secs
+
+    toks_all, secs_all = run(n, cores)
+    n1 = max(1, n // 8)
+    toks_1, secs_1 = run(n1, 1)
+    return {"value": round(toks_all / secs_all, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
+            "sample": f"first {n} of {w.R} rows, all positions ({toks_all} tokens, {secs_all:.1f} s)",
+            "value_1_thread": round(toks_1 / secs_1, 1), "sample_1_thread": f"first {n1} rows ({secs_1:.1f} s)",
+            "trie_build_s": round(build_s, 1)}
+
+
+def run_reference(args):
+    """The oracle as the reference arm: rank 0 only; each step decodes a bounded sample of the
+    workload (the first rows) on the host cores.  The logits come from the stand-in LM (on the GPU
+    when there is one) and are outside the timed region, as in the other arm."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import torch
+
+    import oracle
+    from workloads import make_contexts, make_lm_weights, make_set
+    from workloads.standin_lm import StandInLM
+    w = workload(args)
+    cores = os.cpu_count() or 1
+    dev = "cuda:0" if torch.cuda.is_available() else "cpu"
+    tok, off = make_set(w)
+    t0 = time.time()
+    S = oracle.OracleSet(tok, off, w.V)
+    build_s = time.time() - t0
+    lm = StandInLM(*make_lm_weights(w), w.logits, dev)
+    rows = min(w.R, max(w.K, (args.cpu_sample_rows // w.K) * w.K))
+    B = rows // w.K
+    ctx = make_contexts(w)[:B]
+    seed = 250409135
+
+    def decode():
+        seq = np.full((rows, S.l_max), -1, np.int32)
+        done = np.zeros(rows, np.uint8)
+        logw = np.zeros(rows, np.float64)
+        prev = np.repeat(ctx, w.K).astype(np.int64)
+        secs, toks = 0.0, 0
+        for t in range(S.l_max):
+            if done.all():
+                break
+            hl, dt = logits_to_numpy(lm.logits(torch.as_tensor(prev)))
+            a = time.perf_counter()
+            o = S.step(hl, dt, seq, np.full(rows, t, np.int32), done, seed=seed, step=t, n_threads=cores)
+            secs += time.perf_counter() - a
+            live = done == 0
+            toks += int(live.sum())
+            seq[live, t] = o["token"][live]
+            logw[live] += o["log_mass"][live]
+            prev[live] = o["token"][live]
+            done = np.where(live, o["done"], done).astype(np.uint8)
+        a = time.perf_counter()
+        oracle.resample(logw.reshape(B, w.K).astype(np.float32), seed=seed)
+        secs += time.perf_counter() - a
+        return toks, secs
+
+    for _ in range(min(args.warmup, 1)):
+        decode()
+    toks = secs = 0
+    for _ in range(args.steps):
+        a, b = decode()
+        toks += a
+        secs += b
+    value = toks / secs
+    line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": min(args.warmup, 1), "ms_per_step": round(secs / args.steps * 1e3, 3),
+            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+            "data": "synthetic", "impl": "reference",
+            "config": {"workload": describe(w, S.N), "positions": S.l_max},
+            "cpu_baseline": {"value": round(value, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"first {rows} of {w.R} rows per step, all positions",
+                             "trie_build_s": round(build_s, 1)},
+            "e2e": {"value": round(value, 1), "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    a = parse_args()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

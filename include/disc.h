@@ -1,0 +1,196 @@
+/* disc.h - C ABI of the B200 (sm_100a) DISC + PPV constrained-decoding hot path.
+ *
+ * The library implements the per-step work of the paper "Efficient and Asymptotically Unbiased
+ * Constrained Decoding for Large Language Models" (DISC, Algorithm 1; PPV, Algorithm 2):
+ *
+ *   disc_build_set   Algorithm 2, line 1 ("Prepare") and Section 3.2 "Array Preparation": sort the
+ *                    members of S lexicographically by token id and keep the array on the GPU.
+ *   disc_mask        Algorithm 2, lines 3-7 with M = |V|: the mask of the valid set A_{a,S}
+ *                    (Section 2.1) of a prefix a.
+ *   disc_step        Algorithm 1, lines 5-8 for a batch of partial sequences: mask, sample from
+ *                    P.mask/|P.mask|_1, append, multiply the importance score by |P.mask|_1.
+ *   disc_resample    Algorithm 1, line 22: among K finished candidates pick one with probability
+ *                    x_k / sum_j x_j.
+ *   disc_accept      Algorithm 1, line 16: accept a candidate when x > eps ~ U[0,1].
+ *
+ * Conventions
+ *   - Every function returns 0 (DISC_OK) or a negative DISC_ERR_* code.  Return codes cover
+ *     argument validation and CUDA launch/allocation errors only; problems of a single row are
+ *     reported in that row's status byte and never fail the call.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are memory of the current CUDA
+ *     device, owned by the caller.  `stream` is a cudaStream_t (NULL = the default stream).
+ *   - Except for disc_build_set / disc_free_set / disc_set_info / disc_set_rows, calls only enqueue
+ *     kernels on `stream`: they allocate nothing, do not synchronise the host, and finish in
+ *     stream order.
+ *   - The importance score x of Algorithm 1 is kept as its logarithm `logw` in fp32 (x starts at 1,
+ *     logw at 0; each step adds log |P.mask|_1).
+ *   - The set must be prefix-free (all members of one length, or every member closed by an
+ *     end-of-sequence token that is an ordinary token): "a in S" (Algorithm 1, line 4) is then
+ *     "a's node has no child".
+ *   - Mask layout: W = ceil(V/32) uint32 words per row; token v is bit (v & 31) of word (v >> 5);
+ *     bits at positions >= V are zero.
+ *   - Random numbers: Philox4x32-10, key = (seed low 32 bits, seed high 32 bits).  The uniform of
+ *     output word r is u = ((r >> 9) + 0.5) * 2^-23 (u and 1-u exact in fp32).  Counters:
+ *       sampling  (v >> 2, step, row, 0), word v & 3     one uniform per (row, step, token v)
+ *       resample  (query, 0, 0, 1), word 0
+ *       accept    (query, k, 0, 2), word 0
+ *     where `row` / `query` is row_base / query_base plus the index inside the call.
+ *   - Sampling is Gumbel-max: token = argmax over allowed v of z_v/T - log(-log u_v), lowest id on
+ *     an exact tie; this draws from P.mask/|P.mask|_1.
+ */
+#ifndef DISC_H_
+#define DISC_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define DISC_OK 0
+#define DISC_ERR_ARG (-1)         /* null, negative, out-of-range or misaligned argument          */
+#define DISC_ERR_EMPTY (-2)       /* empty set or empty member                                    */
+#define DISC_ERR_TOKEN (-3)       /* token id outside [0, vocab_size)                             */
+#define DISC_ERR_PREFIX (-4)      /* a member is a proper prefix of another member                */
+#define DISC_ERR_OOM (-5)         /* device or host allocation failed                             */
+#define DISC_ERR_CUDA (-6)        /* a CUDA call failed; see disc_last_cuda_error()               */
+#define DISC_ERR_UNSUPPORTED (-7) /* size or dtype outside what the kernels support               */
+
+/* per-row status bits */
+#define DISC_ROW_DEAD 1     /* prefix / node is not a prefix of any member                        */
+#define DISC_ROW_NOMASS 2   /* allowed probability mass is zero or not finite                     */
+#define DISC_ROW_NONFINITE 4 /* NaN or +Inf among the row's logits (or NaN among the weights)     */
+#define DISC_ROW_DONE 8     /* row was already complete: nothing read, state untouched            */
+
+typedef struct disc_set disc_set_t; /* opaque; owns its device memory */
+
+typedef enum { DISC_F32 = 0, DISC_BF16 = 1 } disc_dtype_t;
+
+#define DISC_MAX_DEPTH 64
+
+typedef struct {
+    int64_t n_members;       /* N: members after de-duplication                                  */
+    int64_t n_entries;       /* E: int32 entries of the sorted table                             */
+    int64_t n_nodes;         /* distinct non-empty prefixes of members (index nodes)             */
+    int32_t vocab_size;      /* V                                                                */
+    int32_t mask_words;      /* W = ceil(V/32)                                                   */
+    int32_t l_max;           /* longest member                                                   */
+    int32_t reserved;
+    int64_t device_bytes;    /* device memory held by the handle                                 */
+    double build_seconds;    /* wall time of disc_build_set                                      */
+    int64_t level_nodes[DISC_MAX_DEPTH]; /* distinct prefixes of length d+1, d = 0..l_max-1      */
+} disc_set_info_t;
+
+/* Build the device-resident constraint array (Algorithm 2, line 1; Section 3.2 "Array
+ * Preparation").
+ *   tokens       host, int32[row_offsets[n_rows]]: the members back to back, in any order
+ *   row_offsets  host, int64[n_rows+1]: member r is tokens[row_offsets[r] .. row_offsets[r+1])
+ *   vocab_size   V; every token must lie in [0, V)
+ *   flags        must be 0
+ *   stream       stream the build kernels run on; the call synchronises it before returning
+ *   out          receives the handle (NULL on error)
+ * The inputs are copied.  Members are sorted lexicographically by token id (a shorter sequence
+ * before its extensions), duplicates are collapsed.  Besides the sorted table the handle holds an
+ * index with one node per distinct non-empty prefix, level by level, from which the valid set of
+ * any prefix is read as a contiguous list.
+ * Errors: DISC_ERR_ARG, DISC_ERR_EMPTY (no member / an empty member), DISC_ERR_TOKEN,
+ * DISC_ERR_PREFIX, DISC_ERR_UNSUPPORTED (n_rows >= 2^31, entries >= 2^32, member longer than
+ * DISC_MAX_DEPTH, V > 4,000,000), DISC_ERR_OOM, DISC_ERR_CUDA. */
+int disc_build_set(const int32_t* tokens, const int64_t* row_offsets, int64_t n_rows,
+                   int32_t vocab_size, uint32_t flags, void* stream, disc_set_t** out);
+
+/* Release the handle and its device memory.  NULL is allowed. */
+void disc_free_set(disc_set_t* s);
+
+/* Sizes of the built set.  `info` is host memory. */
+int disc_set_info(const disc_set_t* s, disc_set_info_t* info);
+
+/* Copy the sorted, de-duplicated table back (the array X of Algorithm 2, without padding).
+ *   tokens_out       host, int32[n_entries]
+ *   row_offsets_out  host, int64[n_members+1]
+ * Synchronises the device. */
+int disc_set_rows(const disc_set_t* s, int32_t* tokens_out, int64_t* row_offsets_out);
+
+/* Start n candidates at the empty sequence (Algorithm 1, line 3: a = [], x = 1).
+ * All arrays are device memory with n entries: node = root, [lo, hi) = [0, N), depth = 0,
+ * logw = 0, done = 0. */
+int disc_state_init(const disc_set_t* s, int64_t n, int32_t* node, int32_t* lo, int32_t* hi,
+                    int32_t* depth, float* logw, uint8_t* done, void* stream);
+
+/* Valid-set masks of n prefixes (Algorithm 2, lines 3-7 in the M = |V| limit; Section 2.1).
+ *   prefix      device, int32[n][prefix_ld]; row i holds prefix_len[i] tokens
+ *   prefix_len  device, int32[n], 0 <= prefix_len[i] <= prefix_ld
+ *   mask_out    device, uint32[n][W] (nullable): bit v set iff prefix+[v] is a prefix of a member
+ *   lo_out, hi_out  device, int32[n] (nullable): the members having the prefix are rows [lo, hi)
+ *               of the sorted table
+ *   node_out    device, int32[n] (nullable): index node of the prefix (the cursor disc_step uses)
+ *   status_out  device, uint8[n]: 0, or DISC_ROW_DEAD when the prefix is a prefix of no member
+ *               (then the mask is zero and lo = hi = node = -1)
+ * A complete member has an empty mask and a range of one row. */
+int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
+              const int32_t* prefix_len, int64_t n, uint32_t* mask_out, int32_t* lo_out,
+              int32_t* hi_out, int32_t* node_out, uint8_t* status_out, void* stream);
+
+/* One decoding step for n candidates (Algorithm 1, lines 5-8; score closed form in Appendix A).
+ *   logits   device, n rows of V values of type `dtype`, row i at element offset i*ld.  The fast
+ *            path needs the base 16-byte aligned and ld*sizeof(value) a multiple of 16; other
+ *            layouts take a slower scalar path.
+ *   inv_temperature  1/T (Algorithm 1's T), finite and > 0
+ *   seed, step, row_base  random-number coordinates (see top of file); `step` must differ between
+ *            the steps of one decode
+ *   node, lo, hi, depth, logw, done   device, in/out state, n entries each
+ *   token_out   device, int32[n]: sampled token, -1 for rows that did nothing
+ *   seq_tokens  device, int32[n][seq_ld] (nullable): the token is also stored at
+ *            seq_tokens[i][depth[i]] (depth before the step) when depth[i] < seq_ld
+ *   logq_out    device, float[n] (nullable): log-probability of the token under the masked,
+ *            renormalised distribution
+ *   logp_out    device, float[n] (nullable): its log-probability under the unmasked distribution
+ *   mask_out    device, uint32[n][W] (nullable): the valid-set mask used by each live row
+ *   status_out  device, uint8[n]
+ * Per live row: z_v = logit_v / T; lse_all = log sum_v e^{z_v}; lse_ok = the same over the valid
+ * set; logw += lse_ok - lse_all; token by Gumbel-max over the valid set; the state moves to the
+ * extended prefix; done is set when the extended prefix is a member.  Rows with done != 0 are
+ * skipped (status DISC_ROW_DONE, token -1, no logits read).  A row whose valid mass is zero keeps
+ * going with the lowest valid token (status DISC_ROW_NOMASS, logw = -inf); NaN/+Inf logits give
+ * status DISC_ROW_NONFINITE and a NaN/Inf logw. */
+int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n,
+              float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base,
+              int32_t* node, int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done,
+              int32_t* token_out, int32_t* seq_tokens, int32_t seq_ld, float* logq_out,
+              float* logp_out, uint32_t* mask_out, uint8_t* status_out, void* stream);
+
+/* K-way importance draw (Algorithm 1, line 22; Appendix A).
+ *   logw        device, float[B][K]: log importance scores of the K candidates of each query
+ *   idx_out     device, int32[B]: chosen candidate, P(k) = x_k / sum_j x_j
+ *   logz_out    device, float[B] (nullable): log((1/K) sum_k x_k), an estimate of log P_L(S)
+ *   seq_tokens  device, int32[B][K][seq_ld] (nullable) and tokens_out device int32[B][seq_ld]
+ *               (nullable): when both are given the chosen candidate's tokens are copied out
+ *   status_out  device, uint8[B]: DISC_ROW_NOMASS when no candidate has a finite positive weight
+ *               (the pick is then uniform), DISC_ROW_NONFINITE when a weight is NaN (it counts as 0)
+ * The pick is the smallest k whose inclusive prefix sum of weights exceeds u * total. */
+int disc_resample(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_t query_base,
+                  int32_t* idx_out, float* logz_out, const int32_t* seq_tokens, int32_t seq_ld,
+                  int32_t* tokens_out, uint8_t* status_out, void* stream);
+
+/* Accept test over K finished candidates per query, in order (Algorithm 1, lines 12-21):
+ *   first_out   device, int32[B]: smallest k with logw[b][k] > log(eps_{b,k}), eps uniform in
+ *               (0,1); -1 when all K candidates are rejected (the caller then falls back to
+ *               disc_resample on K fresh candidates). */
+int disc_accept(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_t query_base,
+                int32_t* first_out, void* stream);
+
+/* Diagnostic: the n sampling uniforms of tokens v0 .. v0+n-1 for (seed, step, row), as fp32.
+ *   out  device, float[n] */
+int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t v0, int32_t n,
+                           float* out, void* stream);
+
+/* Text for a DISC_ERR_* code. */
+const char* disc_error_string(int code);
+
+/* cudaError_t (as int) of the most recent failed CUDA call made by this library on this thread. */
+int disc_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* DISC_H_ */

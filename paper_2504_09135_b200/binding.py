@@ -1,0 +1,296 @@
+"""Thin Python binding of the C ABI in include/disc.h.
+
+Argument marshalling only: every function here checks tensor types, hands raw pointers to the
+CUDA library and returns the output tensors.  torch is used for device memory and streams.  There
+is no CPU fallback: without the compiled library (or without a CUDA device for the calls that need
+one) these functions raise.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+
+import numpy as np
+import torch
+
+from . import build as _build
+
+DISC_F32, DISC_BF16 = 0, 1
+ROW_DEAD, ROW_NOMASS, ROW_NONFINITE, ROW_DONE = 1, 2, 4, 8
+MAX_DEPTH = 64
+
+ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "DISC_ERR_PREFIX",
+          -5: "DISC_ERR_OOM", -6: "DISC_ERR_CUDA", -7: "DISC_ERR_UNSUPPORTED"}
+
+EXPORTS = ["disc_build_set", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
+           "disc_mask", "disc_step", "disc_resample", "disc_accept", "disc_sampling_uniforms",
+           "disc_error_string", "disc_last_cuda_error"]
+
+
+class DiscError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        name = ERRORS.get(code, str(code))
+        extra = ""
+        if code == -6:
+            extra = f" (cudaError {lib().disc_last_cuda_error()})"
+        super().__init__(f"{where} failed: {name}{extra}")
+        self.code = code
+
+
+class _SetInfo(C.Structure):
+    _fields_ = [("n_members", C.c_int64), ("n_entries", C.c_int64), ("n_nodes", C.c_int64),
+                ("vocab_size", C.c_int32), ("mask_words", C.c_int32), ("l_max", C.c_int32),
+                ("reserved", C.c_int32), ("device_bytes", C.c_int64), ("build_seconds", C.c_double),
+                ("level_nodes", C.c_int64 * MAX_DEPTH)]
+
+
+_lib = None
+
+
+def lib():
+    """Load (building first if needed) the CUDA library.  Raises if that is impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.LIB
+    if not os.path.exists(path) or os.path.getmtime(path) < _build._newest_dep():
+        path = _build.build()
+    L = C.CDLL(path)
+    vp, i32, i64, u32, u64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_float
+    L.disc_build_set.argtypes = [vp, vp, i64, i32, u32, vp, C.POINTER(vp)]
+    L.disc_free_set.argtypes = [vp]
+    L.disc_free_set.restype = None
+    L.disc_set_info.argtypes = [vp, C.POINTER(_SetInfo)]
+    L.disc_set_rows.argtypes = [vp, vp, vp]
+    L.disc_state_init.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp]
+    L.disc_mask.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp, vp, vp]
+    L.disc_step.argtypes = [vp, vp, C.c_int, i64, i64, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
+                            vp, vp, i32, vp, vp, vp, vp, vp]
+    L.disc_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, i32, vp, vp, vp]
+    L.disc_accept.argtypes = [vp, i32, i32, u64, i64, vp, vp]
+    L.disc_sampling_uniforms.argtypes = [u64, u32, u32, i32, i32, vp, vp]
+    L.disc_error_string.argtypes = [C.c_int]
+    L.disc_error_string.restype = C.c_char_p
+    L.disc_last_cuda_error.argtypes = []
+    for name in EXPORTS:
+        if name not in ("disc_free_set", "disc_error_string"):
+            getattr(L, name).restype = C.c_int
+    _lib = L
+    return L
+
+
+def _check(rc: int, where: str):
+    if rc != 0:
+        raise DiscError(rc, where)
+
+
+def _stream_ptr(stream=None) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return int(s.cuda_stream)
+
+
+def _dev(t: torch.Tensor, dtype, name: str) -> int:
+    if t is None:
+        return 0
+    if not (isinstance(t, torch.Tensor) and t.is_cuda and t.dtype == dtype and t.is_contiguous()):
+        raise TypeError(f"{name}: expected a contiguous CUDA tensor of {dtype}")
+    return t.data_ptr()
+
+
+class DiscSet:
+    """Handle of a built constraint set (owns device memory; free with .close())."""
+
+    def __init__(self, handle, info: _SetInfo):
+        self._h = handle
+        self.N = int(info.n_members)
+        self.E = int(info.n_entries)
+        self.n_nodes = int(info.n_nodes)
+        self.V = int(info.vocab_size)
+        self.W = int(info.mask_words)
+        self.l_max = int(info.l_max)
+        self.device_bytes = int(info.device_bytes)
+        self.build_seconds = float(info.build_seconds)
+        self.level_nodes = [int(info.level_nodes[d]) for d in range(self.l_max)]
+
+    @property
+    def handle(self):
+        if not self._h:
+            raise RuntimeError("constraint set already freed")
+        return self._h
+
+    def close(self):
+        if getattr(self, "_h", None):
+            lib().disc_free_set(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def disc_build_set(tokens, row_offsets, vocab_size: int, stream=None) -> DiscSet:
+    """tokens int32[E], row_offsets int64[n+1] on the host (numpy or CPU tensors)."""
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    row_offsets = np.ascontiguousarray(row_offsets, dtype=np.int64)
+    if row_offsets.ndim != 1 or row_offsets.shape[0] < 1:
+        raise DiscError(-1, "disc_build_set")
+    if not torch.cuda.is_available():
+        raise RuntimeError("disc_build_set needs a CUDA device; there is no CPU path")
+    h = C.c_void_p()
+    rc = lib().disc_build_set(tokens.ctypes.data, row_offsets.ctypes.data, row_offsets.shape[0] - 1,
+                              int(vocab_size), 0, _stream_ptr(stream), C.byref(h))
+    _check(rc, "disc_build_set")
+    info = _SetInfo()
+    _check(lib().disc_set_info(h, C.byref(info)), "disc_set_info")
+    return DiscSet(h, info)
+
+
+def disc_set_rows(s: DiscSet):
+    tok = np.empty(s.E, dtype=np.int32)
+    off = np.empty(s.N + 1, dtype=np.int64)
+    _check(lib().disc_set_rows(s.handle, tok.ctypes.data, off.ctypes.data), "disc_set_rows")
+    return tok, off
+
+
+@dataclass
+class DiscState:
+    """Per-candidate cursor and importance log-weight, all device tensors of n entries."""
+    node: torch.Tensor
+    lo: torch.Tensor
+    hi: torch.Tensor
+    depth: torch.Tensor
+    logw: torch.Tensor
+    done: torch.Tensor
+
+    @property
+    def n(self) -> int:
+        return self.node.shape[0]
+
+    @staticmethod
+    def empty(n: int, device) -> "DiscState":
+        i32 = dict(dtype=torch.int32, device=device)
+        return DiscState(torch.empty(n, **i32), torch.empty(n, **i32), torch.empty(n, **i32),
+                         torch.empty(n, **i32), torch.empty(n, dtype=torch.float32, device=device),
+                         torch.empty(n, dtype=torch.uint8, device=device))
+
+    def clone(self) -> "DiscState":
+        return DiscState(*(t.clone() for t in (self.node, self.lo, self.hi, self.depth, self.logw, self.done)))
+
+
+def disc_state_init(s: DiscSet, n: int, device="cuda", state: DiscState | None = None, stream=None) -> DiscState:
+    st = DiscState.empty(n, device) if state is None else state
+    rc = lib().disc_state_init(s.handle, n, _dev(st.node, torch.int32, "node"), _dev(st.lo, torch.int32, "lo"),
+                               _dev(st.hi, torch.int32, "hi"), _dev(st.depth, torch.int32, "depth"),
+                               _dev(st.logw, torch.float32, "logw"), _dev(st.done, torch.uint8, "done"),
+                               _stream_ptr(stream))
+    _check(rc, "disc_state_init")
+    return st
+
+
+def disc_mask(s: DiscSet, prefix: torch.Tensor, prefix_len: torch.Tensor, *, want_mask=True, out=None, stream=None):
+    """prefix int32[n, ld], prefix_len int32[n] on the device -> dict(mask, lo, hi, node, status)."""
+    n = prefix_len.shape[0]
+    dev = prefix_len.device
+    ld = prefix.shape[1] if prefix.ndim == 2 else 0
+    if out is None:
+        out = {"mask": torch.empty((n, s.W), dtype=torch.int32, device=dev) if want_mask else None,
+               "lo": torch.empty(n, dtype=torch.int32, device=dev),
+               "hi": torch.empty(n, dtype=torch.int32, device=dev),
+               "node": torch.empty(n, dtype=torch.int32, device=dev),
+               "status": torch.empty(n, dtype=torch.uint8, device=dev)}
+    rc = lib().disc_mask(s.handle, _dev(prefix, torch.int32, "prefix") if ld > 0 else 0, ld,
+                         _dev(prefix_len, torch.int32, "prefix_len"), n,
+                         _dev(out["mask"], torch.int32, "mask"), _dev(out["lo"], torch.int32, "lo"),
+                         _dev(out["hi"], torch.int32, "hi"), _dev(out["node"], torch.int32, "node"),
+                         _dev(out["status"], torch.uint8, "status"), _stream_ptr(stream))
+    _check(rc, "disc_mask")
+    return out
+
+
+@dataclass
+class StepOutputs:
+    token: torch.Tensor
+    status: torch.Tensor
+    logq: torch.Tensor | None = None
+    logp: torch.Tensor | None = None
+    mask: torch.Tensor | None = None
+
+    @staticmethod
+    def empty(n: int, device, *, logq=True, logp=True, mask_words: int = 0) -> "StepOutputs":
+        f = dict(dtype=torch.float32, device=device)
+        return StepOutputs(torch.empty(n, dtype=torch.int32, device=device),
+                           torch.empty(n, dtype=torch.uint8, device=device),
+                           torch.empty(n, **f) if logq else None, torch.empty(n, **f) if logp else None,
+                           torch.empty((n, mask_words), dtype=torch.int32, device=device) if mask_words else None)
+
+
+def disc_step(s: DiscSet, logits: torch.Tensor, state: DiscState, *, inv_temperature=1.0, seed=0, step=0,
+              row_base=0, seq_tokens: torch.Tensor | None = None, out: StepOutputs | None = None,
+              stream=None) -> StepOutputs:
+    """logits [n, ld] float32 or bfloat16 on the device (row stride ld >= V, unit element stride)."""
+    n = state.n
+    if logits.dtype == torch.float32:
+        dt = DISC_F32
+    elif logits.dtype == torch.bfloat16:
+        dt = DISC_BF16
+    else:
+        raise DiscError(-7, "disc_step")
+    if not (logits.is_cuda and logits.ndim == 2 and logits.shape[0] == n and logits.stride(1) == 1):
+        raise TypeError("logits: expected a CUDA tensor [n, >=V] with unit inner stride")
+    ld = logits.stride(0) if n > 1 else max(logits.shape[1], logits.stride(0))
+    if out is None:
+        out = StepOutputs.empty(n, logits.device)
+    seq_ld = 0
+    if seq_tokens is not None:
+        seq_ld = seq_tokens.shape[-1]
+    rc = lib().disc_step(s.handle, logits.data_ptr(), dt, ld, n, float(inv_temperature), int(seed), int(step),
+                         int(row_base), _dev(state.node, torch.int32, "node"), _dev(state.lo, torch.int32, "lo"),
+                         _dev(state.hi, torch.int32, "hi"), _dev(state.depth, torch.int32, "depth"),
+                         _dev(state.logw, torch.float32, "logw"), _dev(state.done, torch.uint8, "done"),
+                         _dev(out.token, torch.int32, "token"), _dev(seq_tokens, torch.int32, "seq_tokens"),
+                         seq_ld, _dev(out.logq, torch.float32, "logq"), _dev(out.logp, torch.float32, "logp"),
+                         _dev(out.mask, torch.int32, "mask"), _dev(out.status, torch.uint8, "status"),
+                         _stream_ptr(stream))
+    _check(rc, "disc_step")
+    return out
+
+
+def disc_resample(logw: torch.Tensor, *, seed=0, query_base=0, seq_tokens: torch.Tensor | None = None,
+                  out=None, stream=None):
+    """logw float32[B, K] on the device -> dict(idx, logz, status, tokens)."""
+    B, K = logw.shape
+    dev = logw.device
+    seq_ld = 0 if seq_tokens is None else seq_tokens.shape[-1]
+    if out is None:
+        out = {"idx": torch.empty(B, dtype=torch.int32, device=dev),
+               "logz": torch.empty(B, dtype=torch.float32, device=dev),
+               "status": torch.empty(B, dtype=torch.uint8, device=dev),
+               "tokens": None if seq_tokens is None else torch.empty((B, seq_ld), dtype=torch.int32, device=dev)}
+    rc = lib().disc_resample(_dev(logw, torch.float32, "logw"), B, K, int(seed), int(query_base),
+                             _dev(out["idx"], torch.int32, "idx"), _dev(out["logz"], torch.float32, "logz"),
+                             _dev(seq_tokens, torch.int32, "seq_tokens"), seq_ld,
+                             _dev(out["tokens"], torch.int32, "tokens"), _dev(out["status"], torch.uint8, "status"),
+                             _stream_ptr(stream))
+    _check(rc, "disc_resample")
+    return out
+
+
+def disc_accept(logw: torch.Tensor, *, seed=0, query_base=0, out=None, stream=None) -> torch.Tensor:
+    B, K = logw.shape
+    if out is None:
+        out = torch.empty(B, dtype=torch.int32, device=logw.device)
+    rc = lib().disc_accept(_dev(logw, torch.float32, "logw"), B, K, int(seed), int(query_base),
+                           _dev(out, torch.int32, "first"), _stream_ptr(stream))
+    _check(rc, "disc_accept")
+    return out
+
+
+def disc_sampling_uniforms(seed: int, step: int, row: int, v0: int, n: int, device="cuda", stream=None):
+    out = torch.empty(n, dtype=torch.float32, device=device)
+    rc = lib().disc_sampling_uniforms(int(seed), int(step), int(row), int(v0), int(n), out.data_ptr(),
+                                      _stream_ptr(stream))
+    _check(rc, "disc_sampling_uniforms")
+    return out

@@ -1,0 +1,90 @@
+// Internal declarations shared by the library's translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "disc.h"
+
+struct disc_set {
+    int32_t V = 0;            // vocabulary size
+    int32_t W = 0;            // mask words per row
+    int32_t l_max = 0;
+    int64_t N = 0;            // members
+    int64_t E = 0;            // table entries
+    int64_t M = 0;            // index nodes including the root (node 0)
+    int device = 0;
+    // sorted table (the array X of Algorithm 2, ragged instead of padded)
+    int32_t* tok = nullptr;        // [E]
+    uint32_t* row_off = nullptr;   // [N+1]
+    // prefix index, breadth-first: node 0 = empty prefix, then all prefixes of length 1, 2, ...
+    // in sorted order.  The children of node j are nodes child_begin[j] .. child_begin[j+1]-1,
+    // ascending in token id.
+    int32_t* node_tok = nullptr;     // [M]   last token of the prefix
+    int32_t* node_lo = nullptr;      // [M]   first table row having the prefix
+    int32_t* child_begin = nullptr;  // [M+1]
+    // first level shortcuts
+    uint32_t* root_mask = nullptr;   // [W]   valid set of the empty prefix
+    int32_t* root_child = nullptr;   // [V]   node of the one-token prefix [v], or -1
+    int64_t level_off[DISC_MAX_DEPTH + 2] = {0};  // node id where level d starts (level_off[0] = 1)
+    int64_t device_bytes = 0;
+    double build_seconds = 0.0;
+};
+
+namespace disc {
+
+extern thread_local int g_last_cuda_error;
+
+inline int cuda_fail(cudaError_t e) {
+    g_last_cuda_error = int(e);
+    return e == cudaErrorMemoryAllocation ? DISC_ERR_OOM : DISC_ERR_CUDA;
+}
+
+#define DISC_CUDA(call)                                         \
+    do {                                                        \
+        cudaError_t e__ = (call);                               \
+        if (e__ != cudaSuccess) return ::disc::cuda_fail(e__);  \
+    } while (0)
+
+// ------------------------------------------------------------------ Philox4x32-10
+// Counter-based generator of Salmon et al. (SC'11).  Round keys depend only on the seed.
+struct PhiloxKey {
+    uint32_t k0, k1;
+};
+
+__host__ __device__ __forceinline__ PhiloxKey philox_key(uint64_t seed) {
+    return PhiloxKey{uint32_t(seed), uint32_t(seed >> 32)};
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               PhiloxKey key) {
+    uint32_t k0 = key.k0, k1 = key.k1;
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = uint64_t(0xD2511F53u) * c0;
+        uint64_t p1 = uint64_t(0xCD9E8D57u) * c2;
+        uint32_t n0 = uint32_t(p1 >> 32) ^ c1 ^ k0;
+        uint32_t n2 = uint32_t(p0 >> 32) ^ c3 ^ k1;
+        c1 = uint32_t(p1);
+        c3 = uint32_t(p0);
+        c0 = n0;
+        c2 = n2;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// top 23 bits k of a word -> u = (2k+1) * 2^-24, exact in fp32, as is 1-u
+__device__ __forceinline__ float uniform_from_bits(uint32_t r) {
+    return float((r >> 9) * 2u + 1u) * 5.9604644775390625e-08f;
+}
+
+__device__ __forceinline__ uint32_t pick_word(const uint4& w, uint32_t lane) {
+    return lane == 0 ? w.x : lane == 1 ? w.y : lane == 2 ? w.z : w.w;
+}
+
+// Gumbel noise -log(-log u) with accurate logarithms
+__device__ __forceinline__ float gumbel_from_uniform(float u) { return -logf(-logf(u)); }
+
+}  // namespace disc

@@ -1,0 +1,68 @@
+"""Decode-loop helper: B queries x K candidates through disc_step, then disc_resample.
+
+Orchestration only (which kernel is enqueued when); all arithmetic is in the CUDA library.  The
+loop never synchronises the host: it runs l_max steps, and rows that finished earlier are skipped
+inside the kernel.
+"""
+from __future__ import annotations
+
+import torch
+
+from .binding import (DiscSet, DiscState, StepOutputs, disc_resample, disc_state_init, disc_step)
+
+
+class DiscDecoder:
+    def __init__(self, s: DiscSet, B: int, K: int, device="cuda", *, want_logq=True, want_logp=True):
+        self.set, self.B, self.K, self.R = s, B, K, B * K
+        self.device = torch.device(device)
+        self.state = DiscState.empty(self.R, self.device)
+        self.out = StepOutputs.empty(self.R, self.device, logq=want_logq, logp=want_logp)
+        self.seq = torch.empty((self.R, s.l_max), dtype=torch.int32, device=self.device)
+        self.res = {"idx": torch.empty(B, dtype=torch.int32, device=self.device),
+                    "logz": torch.empty(B, dtype=torch.float32, device=self.device),
+                    "status": torch.empty(B, dtype=torch.uint8, device=self.device),
+                    "tokens": torch.empty((B, s.l_max), dtype=torch.int32, device=self.device)}
+
+    def reset(self):
+        self.seq.fill_(-1)
+        disc_state_init(self.set, self.R, state=self.state)
+
+    def step(self, logits: torch.Tensor, step: int, *, seed=0, inv_temperature=1.0, row_base=0) -> StepOutputs:
+        return disc_step(self.set, logits, self.state, inv_temperature=inv_temperature, seed=seed, step=step,
+                         row_base=row_base, seq_tokens=self.seq, out=self.out)
+
+    def finish(self, *, seed=0, query_base=0):
+        return disc_resample(self.state.logw.view(self.B, self.K), seed=seed, query_base=query_base,
+                             seq_tokens=self.seq.view(self.B, self.K, -1), out=self.res)
+
+    def decode(self, lm, ctx: torch.Tensor, *, seed=0, inv_temperature=1.0, keep_logits=None):
+        """Free-running decode: `lm.logits(prev)` gives the [R, V] logits after tokens `prev`.
+
+        ctx: int tensor [B], the context token of each query.  keep_logits: optional list that
+        receives each step's logits tensor (for replay)."""
+        self.reset()
+        prev = ctx.to(self.device, torch.int64).repeat_interleave(self.K)
+        for t in range(self.set.l_max):
+            logits = lm.logits(prev)
+            if keep_logits is not None:
+                keep_logits.append(logits)
+            o = self.step(logits, t, seed=seed, inv_temperature=inv_temperature)
+            prev = torch.where(o.token >= 0, o.token.to(torch.int64), prev)
+        return self.finish(seed=seed)
+
+    def replay(self, logits_per_step, *, seed=0, inv_temperature=1.0):
+        """Decode over logits that are already resident on the device, one tensor per step."""
+        self.reset()
+        for t, logits in enumerate(logits_per_step):
+            self.step(logits, t, seed=seed, inv_temperature=inv_temperature)
+        return self.finish(seed=seed)
+
+    def replay_from_host(self, host_logits_per_step, staging: torch.Tensor, *, seed=0, inv_temperature=1.0):
+        """Same decode with every step's logits copied from (pinned) host memory first, and the
+        result read back to the host at the end."""
+        self.reset()
+        for t, h in enumerate(host_logits_per_step):
+            staging.copy_(h, non_blocking=True)
+            self.step(staging, t, seed=seed, inv_temperature=inv_temperature)
+        r = self.finish(seed=seed)
+        return {"idx": r["idx"].cpu(), "tokens": r["tokens"].cpu(), "logz": r["logz"].cpu()}
