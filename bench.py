@@ -39,14 +39,18 @@ NCU_TRAFFIC_RATIO = None
 def parse_args():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="large", choices=["tiny", "genret", "llm", "large"])
-    ap.add_argument("--draws", type=int, default=0, help="override the number of members drawn (debugging)")
+    ap.add_argument("--draws", type=int, default=0, help="override the number of members drawn (profiling)")
+    ap.add_argument("--B", type=int, default=0, help="override the number of queries (profiling)")
+    ap.add_argument("--K", type=int, default=0, help="override the candidates per query (profiling)")
+    ap.add_argument("--positions", type=int, default=0,
+                    help="decode only the first P token positions (profiling: bounds the resident logits)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
-    ap.add_argument("--cpu-sample-rows", type=int, default=256)
+    ap.add_argument("--cpu-sample-rows", type=int, default=4096)
     return ap.parse_args()
 
 
@@ -90,7 +94,7 @@ class ClockSampler:
                         self.reasons.add(k)
             except Exception:
                 pass
-            self._stop.wait(0.02)
+            self._stop.wait(0.004)
 
     def start(self):
         if self.nv is not None:
@@ -133,10 +137,14 @@ def logits_to_numpy(t):
 
 def workload(args):
     from workloads import CONFIGS, scaled
-    w = CONFIGS[args.workload]
+    over = {}
     if args.draws:
-        w = scaled(args.workload, n_draws=args.draws)
-    return w
+        over["n_draws"] = args.draws
+    if args.B:
+        over["B"] = args.B
+    if args.K:
+        over["K"] = args.K
+    return scaled(args.workload, **over) if over else CONFIGS[args.workload]
 
 
 def describe(w, N=None):
@@ -176,7 +184,7 @@ def run_ours(args):
     ctx = torch.as_tensor(make_contexts(w, salt=rank), device=dev)
     dec = disc.DiscDecoder(G, w.B, w.K, dev)
     seed = 250409135 + rank
-    L = G.l_max
+    L = min(G.l_max, args.positions) if args.positions else G.l_max
     esize = 4 if w.logits == "f32" else 2
 
     # ---- recording decode: keep every position's logits; count live rows and valid-set sizes
@@ -201,7 +209,7 @@ def run_ours(args):
     first_tokens = first["tokens"].clone()
     first_logw = dec.state.logw.clone()
     torch.cuda.synchronize()
-    assert bool(dec.state.done.all()), "decode did not finish within l_max steps"
+    assert args.positions or bool(dec.state.done.all()), "decode did not finish within l_max steps"
     del mask_buf, probe
     tokens_per_decode = int(sum(alive))
     launches = [t for t in range(L) if alive[t] > 0]
@@ -382,7 +390,7 @@ def cpu_baseline(w, tok, off, logits_rows, seq, seed):
         return toks, secs
 
     toks_all, secs_all = run(n, cores)
-    n1 = max(1, n // 8)
+    n1 = max(1, n // 16)
     toks_1, secs_1 = run(n1, 1)
     return {"value": round(toks_all / secs_all, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
             "sample": f"first {n} of {w.R} rows, all positions ({toks_all} tokens, {secs_all:.1f} s)",
@@ -411,7 +419,7 @@ def run_reference(args):
     S = oracle.OracleSet(tok, off, w.V)
     build_s = time.time() - t0
     lm = StandInLM(*make_lm_weights(w), w.logits, dev)
-    rows = min(w.R, max(w.K, (args.cpu_sample_rows // w.K) * w.K))
+    rows = min(w.R, max(w.K, (min(args.cpu_sample_rows, 512) // w.K) * w.K))
     B = rows // w.K
     ctx = make_contexts(w)[:B]
     seed = 250409135

@@ -61,6 +61,8 @@ extern "C" {
 #define DISC_ROW_NOMASS 2   /* allowed probability mass is zero or not finite                     */
 #define DISC_ROW_NONFINITE 4 /* NaN or +Inf among the row's logits (or NaN among the weights)     */
 #define DISC_ROW_DONE 8     /* row was already complete: nothing read, state untouched            */
+#define DISC_ROW_FAULT 16   /* an asynchronous copy inside the kernel never completed (bounded wait
+                               gave up); the row's state is untouched                             */
 
 typedef struct disc_set disc_set_t; /* opaque; owns its device memory */
 
@@ -75,7 +77,7 @@ typedef struct {
     int32_t vocab_size;      /* V                                                                */
     int32_t mask_words;      /* W = ceil(V/32)                                                   */
     int32_t l_max;           /* longest member                                                   */
-    int32_t reserved;
+    int32_t n_heavy;         /* nodes with more than 1024 children (their masks are prebuilt)    */
     int64_t device_bytes;    /* device memory held by the handle                                 */
     double build_seconds;    /* wall time of disc_build_set                                      */
     int64_t level_nodes[DISC_MAX_DEPTH]; /* distinct prefixes of length d+1, d = 0..l_max-1      */

@@ -9,6 +9,7 @@ The shared object is compiled on first use with g++ (a few seconds).
 from __future__ import annotations
 
 import ctypes as C
+import hashlib
 import os
 import subprocess
 
@@ -24,12 +25,20 @@ F32, BF16 = 0, 1
 
 def build(force: bool = False) -> str:
     """Compile the oracle if the shared object is missing or older than the source."""
-    stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+    with open(_SRC, "rb") as f:
+        digest = hashlib.sha256(f.read()).hexdigest()
+    try:
+        with open(_LIB + ".sha256") as f:
+            stale = (not os.path.exists(_LIB)) or f.read().strip() != digest
+    except OSError:
+        stale = True
     if force or stale:
         tmp = _LIB + f".tmp{os.getpid()}"
         subprocess.run(["g++", "-O2", "-std=c++17", "-fPIC", "-shared", "-pthread", "-o", tmp, _SRC],
                        check=True)
         os.replace(tmp, _LIB)
+        with open(_LIB + ".sha256", "w") as f:
+            f.write(digest)
     return _LIB
 
 

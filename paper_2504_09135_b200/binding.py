@@ -17,7 +17,7 @@ import torch
 from . import build as _build
 
 DISC_F32, DISC_BF16 = 0, 1
-ROW_DEAD, ROW_NOMASS, ROW_NONFINITE, ROW_DONE = 1, 2, 4, 8
+ROW_DEAD, ROW_NOMASS, ROW_NONFINITE, ROW_DONE, ROW_FAULT = 1, 2, 4, 8, 16
 MAX_DEPTH = 64
 
 ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "DISC_ERR_PREFIX",
@@ -41,7 +41,7 @@ class DiscError(RuntimeError):
 class _SetInfo(C.Structure):
     _fields_ = [("n_members", C.c_int64), ("n_entries", C.c_int64), ("n_nodes", C.c_int64),
                 ("vocab_size", C.c_int32), ("mask_words", C.c_int32), ("l_max", C.c_int32),
-                ("reserved", C.c_int32), ("device_bytes", C.c_int64), ("build_seconds", C.c_double),
+                ("n_heavy", C.c_int32), ("device_bytes", C.c_int64), ("build_seconds", C.c_double),
                 ("level_nodes", C.c_int64 * MAX_DEPTH)]
 
 
@@ -53,9 +53,7 @@ def lib():
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.LIB
-    if not os.path.exists(path) or os.path.getmtime(path) < _build._newest_dep():
-        path = _build.build()
+    path = _build.LIB if _build.is_fresh() else _build.build()
     L = C.CDLL(path)
     vp, i32, i64, u32, u64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_float
     L.disc_build_set.argtypes = [vp, vp, i64, i32, u32, vp, C.POINTER(vp)]
@@ -109,6 +107,7 @@ class DiscSet:
         self.V = int(info.vocab_size)
         self.W = int(info.mask_words)
         self.l_max = int(info.l_max)
+        self.n_heavy = int(info.n_heavy)
         self.device_bytes = int(info.device_bytes)
         self.build_seconds = float(info.build_seconds)
         self.level_nodes = [int(info.level_nodes[d]) for d in range(self.l_max)]

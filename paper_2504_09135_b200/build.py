@@ -6,6 +6,7 @@ The result, paper_2504_09135_b200/libdisc_b200.so, exports the C ABI declared in
 """
 from __future__ import annotations
 
+import hashlib
 import os
 import subprocess
 import sys
@@ -17,6 +18,7 @@ CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(ROOT, "include")
 OBJ_DIR = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libdisc_b200.so")
+STAMP = LIB + ".sha256"
 
 SOURCES = ["disc_build.cu", "disc_mask.cu", "disc_step.cu", "disc_resample.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
@@ -30,13 +32,25 @@ def _nvcc() -> str:
     raise RuntimeError("nvcc not found")
 
 
-def _newest_dep() -> float:
-    deps = [os.path.join(CSRC, f) for f in os.listdir(CSRC)] + [os.path.join(INCLUDE, "disc.h")]
-    return max(os.path.getmtime(d) for d in deps)
+def source_hash() -> str:
+    """Digest of every source the library is built from (file times do not survive a copy)."""
+    h = hashlib.sha256(" ".join(NVCC_FLAGS[:8]).encode())
+    for path in sorted(os.path.join(CSRC, f) for f in os.listdir(CSRC)) + [os.path.join(INCLUDE, "disc.h")]:
+        with open(path, "rb") as f:
+            h.update(os.path.basename(path).encode() + b"\0" + f.read())
+    return h.hexdigest()
+
+
+def is_fresh() -> bool:
+    try:
+        with open(STAMP) as f:
+            return os.path.exists(LIB) and f.read().strip() == source_hash()
+    except OSError:
+        return False
 
 
 def build(force: bool = False, verbose: bool = False) -> str:
-    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= _newest_dep():
+    if not force and is_fresh():
         return LIB
     os.makedirs(OBJ_DIR, exist_ok=True)
     nvcc = _nvcc()
@@ -57,6 +71,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
     tmp = LIB + f".tmp{os.getpid()}"
     subprocess.run([nvcc, "-shared", "-o", tmp, *objs, "-gencode", "arch=compute_100a,code=sm_100a"], check=True)
     os.replace(tmp, LIB)
+    with open(STAMP, "w") as f:
+        f.write(source_hash())
     return LIB
 
 

@@ -168,6 +168,24 @@ __global__ void k_root_tables(const int32_t* __restrict__ node_tok, int64_t firs
     atomicOr(&root_mask[t >> 5], 1u << (t & 31));
 }
 
+struct HeavyPred {
+    const int32_t* child_begin;
+    __device__ bool operator()(int32_t j) const {
+        return j > 0 && (child_begin[j + 1] - child_begin[j]) > DISC_HEAVY_MIN;
+    }
+};
+
+// one block per heavy node: set the bits of its children in its prebuilt mask row
+__global__ void k_heavy_masks(const int32_t* __restrict__ heavy_nodes, const int32_t* __restrict__ child_begin,
+                              const int32_t* __restrict__ node_tok, int32_t W, uint32_t* __restrict__ masks) {
+    const int32_t j = heavy_nodes[blockIdx.x];
+    uint32_t* row = masks + size_t(blockIdx.x) * W;
+    for (int32_t i = child_begin[j] + threadIdx.x; i < child_begin[j + 1]; i += blockDim.x) {
+        int32_t t = node_tok[i];
+        atomicOr(&row[t >> 5], 1u << (t & 31));
+    }
+}
+
 __global__ void k_fill_i32(int32_t* p, int32_t v, int64_t n) {
     int64_t i = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (i < n) p[i] = v;
@@ -368,8 +386,39 @@ int build_impl(const int32_t* tokens, const int64_t* row_offsets, int64_t n, int
     DISC_CUDA(cudaGetLastError());
     DISC_CUDA(cudaStreamSynchronize(st));
 
+    // ---- prebuilt masks of heavy nodes (each has more than DISC_HEAVY_MIN children, so there are
+    // fewer than M / DISC_HEAVY_MIN of them)
+    DevBuf heavy_nodes, heavy_masks, n_sel;
+    {
+        const int64_t cap = M / DISC_HEAVY_MIN + 1;
+        DISC_CUDA(heavy_nodes.alloc(size_t(cap) * 4));
+        DISC_CUDA(n_sel.alloc(8));
+        cub::CountingInputIterator<int32_t> ids(0);
+        HeavyPred pred{child_begin.as<int32_t>()};
+        size_t need = 0;
+        DISC_CUDA(cub::DeviceSelect::If(nullptr, need, ids, heavy_nodes.as<int32_t>(), n_sel.as<int32_t>(), int(M),
+                                        pred, st));
+        if (need > temp.bytes) DISC_CUDA(temp.alloc(need));
+        DISC_CUDA(cub::DeviceSelect::If(temp.p, need, ids, heavy_nodes.as<int32_t>(), n_sel.as<int32_t>(), int(M),
+                                        pred, st));
+        int32_t H = 0;
+        DISC_CUDA(cudaMemcpyAsync(&H, n_sel.p, 4, cudaMemcpyDeviceToHost, st));
+        DISC_CUDA(cudaStreamSynchronize(st));
+        S->n_heavy = H;
+        DISC_CUDA(heavy_masks.alloc(size_t(H > 0 ? H : 1) * size_t(S->W) * 4));
+        if (H > 0) {
+            DISC_CUDA(cudaMemsetAsync(heavy_masks.p, 0, size_t(H) * size_t(S->W) * 4, st));
+            k_heavy_masks<<<unsigned(H), 256, 0, st>>>(heavy_nodes.as<int32_t>(), child_begin.as<int32_t>(),
+                                                     node_tok.as<int32_t>(), S->W, heavy_masks.as<uint32_t>());
+            DISC_CUDA(cudaGetLastError());
+            DISC_CUDA(cudaStreamSynchronize(st));
+        }
+    }
+
     S->device_bytes = int64_t(tok.bytes + row_off.bytes + node_tok.bytes + node_lo.bytes + child_begin.bytes +
-                              root_mask.bytes + root_child.bytes);
+                              root_mask.bytes + root_child.bytes + heavy_nodes.bytes + heavy_masks.bytes);
+    S->heavy_nodes = static_cast<int32_t*>(heavy_nodes.take());
+    S->heavy_masks = static_cast<uint32_t*>(heavy_masks.take());
     S->tok = static_cast<int32_t*>(tok.take());
     S->row_off = static_cast<uint32_t*>(row_off.take());
     S->node_tok = static_cast<int32_t*>(node_tok.take());
@@ -414,6 +463,8 @@ void disc_free_set(disc_set_t* s) {
     cudaFree(s->child_begin);
     cudaFree(s->root_mask);
     cudaFree(s->root_child);
+    cudaFree(s->heavy_nodes);
+    cudaFree(s->heavy_masks);
     delete s;
 }
 
@@ -426,6 +477,7 @@ int disc_set_info(const disc_set_t* s, disc_set_info_t* info) {
     info->vocab_size = s->V;
     info->mask_words = s->W;
     info->l_max = s->l_max;
+    info->n_heavy = s->n_heavy;
     info->device_bytes = s->device_bytes;
     info->build_seconds = s->build_seconds;
     for (int d = 0; d < s->l_max; ++d) info->level_nodes[d] = s->level_off[d + 1] - s->level_off[d];

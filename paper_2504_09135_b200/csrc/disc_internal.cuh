@@ -26,14 +26,34 @@ struct disc_set {
     // first level shortcuts
     uint32_t* root_mask = nullptr;   // [W]   valid set of the empty prefix
     int32_t* root_child = nullptr;   // [V]   node of the one-token prefix [v], or -1
+    // prebuilt masks of the nodes with more than DISC_HEAVY_MIN children ("heavy" nodes)
+    int32_t n_heavy = 0;
+    int32_t* heavy_nodes = nullptr;  // [n_heavy] ascending node ids
+    uint32_t* heavy_masks = nullptr; // [n_heavy][W]
     int64_t level_off[DISC_MAX_DEPTH + 2] = {0};  // node id where level d starts (level_off[0] = 1)
     int64_t device_bytes = 0;
     double build_seconds = 0.0;
 };
 
+// a node with more children than this has its valid-set mask prebuilt at set-build time
+#define DISC_HEAVY_MIN 1024
+
 namespace disc {
 
 extern thread_local int g_last_cuda_error;
+
+// index of `node` in the ascending list of heavy nodes, or -1 (one thread; the list is small)
+__device__ __forceinline__ int32_t heavy_index(const int32_t* __restrict__ heavy_nodes, int32_t n_heavy,
+                                               int32_t node) {
+    int32_t a = 0, b = n_heavy;
+    while (a < b) {
+        int32_t m = (a + b) >> 1;
+        int32_t v = __ldg(heavy_nodes + m);
+        if (v == node) return m;
+        if (v < node) a = m + 1; else b = m;
+    }
+    return -1;
+}
 
 inline int cuda_fail(cudaError_t e) {
     g_last_cuda_error = int(e);

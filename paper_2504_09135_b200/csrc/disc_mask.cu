@@ -3,8 +3,9 @@
 // One warp per prefix.  The warp walks the prefix down the index: the first token goes through a
 // direct table, every further token is located among the current node's sorted children by
 // warp-cooperative range narrowing (32 probes per round).  The node's children are the valid set
-// (Section 2.1); the warp then writes the packed mask row: a 16-byte zero fill of the row followed
-// by the few set words (the empty prefix copies a prebuilt row instead).
+// (Section 2.1).  The warp then writes the packed mask row with 16-byte stores: a copy of the
+// prebuilt row for the empty prefix and for nodes with many children, otherwise a zero fill
+// followed by the few set words.
 
 #include "disc_internal.cuh"
 
@@ -21,9 +22,9 @@ struct MaskParams {
     uint32_t* mask_out;
     int32_t *lo_out, *hi_out, *node_out;
     uint8_t* status_out;
-    const int32_t *node_tok, *node_lo, *child_begin, *root_child;
-    const uint32_t* root_mask;
-    int32_t V, W, N;
+    const int32_t *node_tok, *node_lo, *child_begin, *root_child, *heavy_nodes;
+    const uint32_t *root_mask, *heavy_masks;
+    int32_t V, W, N, n_heavy;
 };
 
 __device__ __forceinline__ int32_t find_child(const int32_t* __restrict__ node_tok, int32_t cb, int32_t ce, int32_t t,
@@ -43,6 +44,11 @@ __device__ __forceinline__ int32_t find_child(const int32_t* __restrict__ node_t
     bool eq = (i < b) && (__ldg(node_tok + i) == t);
     uint32_t bal = __ballot_sync(0xffffffffu, eq);
     return bal ? a + (__ffs(bal) - 1) : -1;
+}
+
+__device__ __forceinline__ void st_stream16(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
 }
 
 template <bool VEC>
@@ -79,18 +85,30 @@ __global__ void __launch_bounds__(MASK_THREADS) disc_mask_kernel(const MaskParam
         }
         if (!p.mask_out) continue;
 
+        // source row: prebuilt (root or heavy node) or zeros
+        const uint32_t* src = nullptr;
+        if (ok && node == 0) src = p.root_mask;
+        else if (ok && ce - cb > DISC_HEAVY_MIN) {
+            const int32_t h = disc::heavy_index(p.heavy_nodes, p.n_heavy, node);
+            if (h >= 0) src = p.heavy_masks + size_t(h) * p.W;
+        }
         uint32_t* row = p.mask_out + size_t(i) * p.W;
-        const bool copy_root = ok && node == 0;
         if (VEC) {
             uint4* row4 = reinterpret_cast<uint4*>(row);
-            const uint4* src4 = reinterpret_cast<const uint4*>(p.root_mask);
+            const uint4* src4 = reinterpret_cast<const uint4*>(src);
             const int n4 = p.W >> 2;
-            for (int w = lane; w < n4; w += 32) row4[w] = copy_root ? __ldg(src4 + w) : make_uint4(0u, 0u, 0u, 0u);
-            for (int w = (n4 << 2) + lane; w < p.W; w += 32) row[w] = copy_root ? __ldg(p.root_mask + w) : 0u;
+            if (src) {
+                for (int w = lane; w < n4; w += 32) st_stream16(row4 + w, __ldg(src4 + w));
+                for (int w = (n4 << 2) + lane; w < p.W; w += 32) row[w] = __ldg(src + w);
+            } else {
+                const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+                for (int w = lane; w < n4; w += 32) row4[w] = z;
+                for (int w = (n4 << 2) + lane; w < p.W; w += 32) row[w] = 0u;
+            }
         } else {
-            for (int w = lane; w < p.W; w += 32) row[w] = copy_root ? __ldg(p.root_mask + w) : 0u;
+            for (int w = lane; w < p.W; w += 32) row[w] = src ? __ldg(src + w) : 0u;
         }
-        if (!ok || copy_root) continue;
+        if (!ok || src) continue;
         __syncwarp();   // the zero fill is ordered before this warp's bit updates
         for (int32_t j = cb + lane; j < ((ce - cb + 31) / 32) * 32 + cb; j += 32) {
             const bool have = j < ce;
@@ -118,6 +136,7 @@ extern "C" int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t pre
     p.mask_out = mask_out; p.lo_out = lo_out; p.hi_out = hi_out; p.node_out = node_out; p.status_out = status_out;
     p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
     p.root_child = s->root_child; p.root_mask = s->root_mask;
+    p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
     p.V = s->V; p.W = s->W; p.N = int32_t(s->N);
 
     int dev = 0, sms = 0;

@@ -2,13 +2,27 @@
 // valid-set lookup, masked and unmasked log-sum-exp over the V logits, Gumbel-max sampling,
 // importance log-weight update and the move of the row's cursor to the extended prefix.
 //
-// One thread block per row.  The row's V logits are streamed once with 16-byte loads; each
-// thread accumulates sum 2^(z*log2e/T - ref) against its own reference (the maximum of the first
-// vector it sees), which keeps the inner loop at one FMA, one ex2 and one add per logit.  The
-// valid set comes from the prefix index as a contiguous child list.  Rows with few children gather
-// their logits directly ("gather path"); rows with many children turn the list into a bitmask in
-// shared memory that the streaming loop consults ("dense path").  A row whose fast sums are not
-// finite, or whose valid mass underflowed, is redone by a plain two-pass routine ("careful path").
+// One thread block per row.
+//   * Streaming.  The row's logits are pulled into a shared-memory ring by bulk asynchronous
+//     copies (cp.async.bulk + mbarrier, one elected thread issues them), so several chunks are in
+//     flight per block whatever the register budget; rows that are not 16-byte aligned take a
+//     plain scalar-load path.
+//   * Sums.  Each thread accumulates sum 2^(x*c - ref) against its own reference (the maximum of
+//     the first vector it sees), c = log2(e)/T: one FMA, one ex2 and one add per logit.  Partial
+//     sums are kept as (m, s) pairs meaning 2^m * s and merged exactly.  All differences are formed
+//     between references before any large value is added, so a common offset of the logits does
+//     not cost accuracy.
+//   * Valid set.  The prefix index gives the row's children as a contiguous list.  Rows with at
+//     most DISC_HEAVY_MIN children gather their few logits directly ("gather path").  Rows with
+//     more use a bitmask in shared memory (prebuilt at set-build time) that the streaming loop
+//     consults ("dense path").
+//   * Sampling.  token = argmax over allowed v of (x_v - xref)/T + g_v with g_v = -log(-log u_v),
+//     u_v from Philox4x32-10 keyed by (token, step, row).  In the dense path a token is evaluated
+//     exactly only if it can still win: with w = 1 - u, g > t implies w < e^-t, so a token whose
+//     w is at least e^(z - best) (times a safety factor) is skipped without taking a logarithm;
+//     e^(z - best) is the already computed 2^(x*c - ref) times a per-thread constant.
+//   * A row whose fast sums are not finite, or that lost an allowed term to underflow, is redone
+//     by a plain two-pass routine with exact scores ("careful path").
 
 #include <math_constants.h>
 
@@ -20,10 +34,15 @@ using namespace disc;
 
 constexpr int STEP_THREADS = 256;
 constexpr int STEP_WARPS = STEP_THREADS / 32;
-constexpr int GATHER_MAX = 1024;   // rows with at most this many children skip the bitmask
-constexpr int UNROLL = 4;
+constexpr int CHUNK_BYTES = 8192;                       // one ring stage
+constexpr int STAGES = 4;
+constexpr int VPT = CHUNK_BYTES / 16 / STEP_THREADS;    // 16-byte vectors per thread and stage
+constexpr int RING_BYTES = CHUNK_BYTES * STAGES;
+constexpr uint64_t WAIT_LIMIT_NS = 250ull * 1000 * 1000;  // an mbarrier wait gives up after 0.25 s
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
+constexpr float SAFETY = 1.0009765625f;                 // 1 + 2^-10 on the skip bound
+constexpr float TWO_M24 = 5.9604644775390625e-08f;      // 2^-24: smallest possible w
 
 struct StepParams {
     const void* logits;
@@ -45,9 +64,9 @@ struct StepParams {
     uint32_t* mask_out;
     uint8_t* status_out;
     // set
-    const int32_t *node_tok, *node_lo, *child_begin, *root_child;
-    const uint32_t* root_mask;
-    int32_t V, W;
+    const int32_t *node_tok, *node_lo, *child_begin, *root_child, *heavy_nodes;
+    const uint32_t *root_mask, *heavy_masks;
+    int32_t V, W, n_heavy;
     int64_t M;
 };
 
@@ -81,12 +100,48 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-__device__ __forceinline__ uint4 ld_stream16(const void* p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
+// ---- mbarrier / bulk-copy wrappers -------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ uint64_t global_ns() {
+    uint64_t t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: gives up (returns false) after WAIT_LIMIT_NS without the phase completing.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
+    const uint64_t t0 = global_ns();
+    while (!mbar_try_wait(bar, parity)) {
+        if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
+    }
+    return true;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
+    return mbar_try_wait(bar, parity) ? true : mbar_wait_slow(bar, parity);
+}
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
+                 "l"(src), "r"(bytes), "r"(bar)
+                 : "memory");
 }
 
 template <int DT>
@@ -118,11 +173,6 @@ struct Elem<DISC_BF16> {
     }
 };
 
-struct RowRng {
-    PhiloxKey key;
-    uint32_t step, row;
-};
-
 // Gumbel-perturbed score of a token with raw logit x, relative to the row's reference logit xref.
 // The argmax does not depend on the common shift, and subtracting before scaling keeps the score
 // accurate to a few ulp of (x - xref) whatever offset the logits carry.
@@ -130,11 +180,100 @@ __device__ __forceinline__ float gumbel_score(float x, float xref, float inv_t, 
     return (x - xref) * inv_t + gumbel_from_uniform(uniform_from_bits(word));
 }
 
-__device__ __forceinline__ void consider(Best& b, float score, int32_t tok, int32_t child) {
+// w = 1 - u of a random word, exact: with k' the complement of the word's top 23 bits,
+// w = (2k'+1) * 2^-24.  No integer-to-float conversion is needed: 1.k' - (1 - 2^-24).
+__device__ __forceinline__ float complement_uniform(uint32_t word) {
+    return __uint_as_float(0x3f800000u | ((~word) >> 9)) - 0.99999994039535522f;
+}
+
+// Per-thread accumulators of the streaming loop.
+struct Acc {
+    float mref = 0.f;        // reference exponent (log2 domain) of this thread's sums
+    float s_all0 = 0.f, s_all1 = 0.f;
+    float s_ok = 0.f;
+    bool touched = false;
+    bool lost = false;       // an allowed term underflowed to zero against mref
+    // sampling
+    Best best{-__builtin_huge_valf(), -1, -1};
+    float cbound = __builtin_huge_valf();   // SAFETY * 2^(mref - xref*c - best*log2e): e * cbound bounds e^(z - best)
+};
+
+struct RowCtx {
+    float c2, inv_t, xref;
+    PhiloxKey key;
+    uint32_t step, row;
+};
+
+__device__ __forceinline__ void set_reference(Acc& a, const RowCtx& r, float xmax) {
+    const float m = xmax * r.c2;
+    a.mref = (fabsf(m) < CUDART_INF_F) ? m : 0.f;
+    a.touched = true;
+}
+
+__device__ __forceinline__ void update_bound(Acc& a, const RowCtx& r) {
+    // exponent of e^(z - best) / 2^(x*c - mref); fma keeps (mref - xref*c) exact to one rounding
+    a.cbound = SAFETY * exp2f(fmaf(-r.xref, r.c2, a.mref) - a.best.score * LOG2E_F);
+}
+
+__device__ __forceinline__ void exact_candidate(Acc& a, const RowCtx& r, float x, uint32_t word, int32_t v) {
     // Tokens arrive in ascending order inside a thread, so strict '>' keeps the lowest id on a
     // tie.  NaN and -inf scores never win; a row without any finite score falls back to its
     // lowest valid token at the end.
-    if (score > b.score) { b.score = score; b.tok = tok; b.child = child; }
+    const float score = gumbel_score(x, r.xref, r.inv_t, word);
+    if (score > a.best.score) {
+        a.best.score = score; a.best.tok = v; a.best.child = -1;
+        update_bound(a, r);
+    }
+}
+
+// one vector of EPV logits starting at token v0
+template <int EPV, bool DENSE>
+__device__ __forceinline__ void consume(Acc& a, const RowCtx& r, const float (&x)[EPV], int v0,
+                                        const uint32_t* __restrict__ smask) {
+    float e[EPV];
+#pragma unroll
+    for (int j = 0; j < EPV; ++j) e[j] = ex2_approx(fmaf(x[j], r.c2, -a.mref));
+#pragma unroll
+    for (int j = 0; j < EPV; j += 2) {
+        a.s_all0 += e[j];
+        if (j + 1 < EPV) a.s_all1 += e[j + 1];
+    }
+    if constexpr (DENSE) {
+        const uint32_t bits = (smask[v0 >> 5] >> (v0 & 31)) & ((1u << EPV) - 1u);
+        if (bits) {
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) {
+                const bool on = (bits >> j) & 1u;
+                a.s_ok += on ? e[j] : 0.f;
+                a.lost |= on && !(e[j] > 0.f);
+            }
+#pragma unroll
+            for (int q = 0; q < (EPV + 3) / 4; ++q) {
+                const uint32_t nib = (bits >> (4 * q)) & 0xFu;
+                if (nib) {
+                    // no token of this group can win if even the largest noise is not enough:
+                    // w >= 2^-24 always, so e*cbound < 2^-24 for all four means "skip" without
+                    // drawing the random numbers
+                    float emax = e[4 * q];
+#pragma unroll
+                    for (int l = 1; l < (EPV < 4 ? EPV : 4); ++l) emax = fmaxf(emax, e[4 * q + l]);
+                    if (!(emax * a.cbound < TWO_M24)) {
+                        const uint4 w4 = philox4x32_10(uint32_t(v0 >> 2) + q, r.step, r.row, 0u, r.key);
+#pragma unroll
+                        for (int l = 0; l < (EPV < 4 ? EPV : 4); ++l) {
+                            if ((nib >> l) & 1u) {
+                                const int j = 4 * q + l;
+                                const int v = v0 + j;
+                                const uint32_t word = pick_word(w4, v & 3);
+                                if (!(complement_uniform(word) >= e[j] * a.cbound))
+                                    exact_candidate(a, r, x[j], word, v);
+                            }
+                        }
+                    }
+                }
+            }
+        }
+    }
 }
 
 // ---- block-wide helpers -----------------------------------------------------------------------
@@ -169,10 +308,21 @@ __device__ float block_sum(float v, float* scratch) {
     return r;
 }
 
-// Valid set of `node` as a bitmask in shared memory (all threads of the block).
-__device__ void build_mask(uint32_t* smask, const StepParams& p, int32_t node, int32_t cb, int32_t ce) {
+// Valid set of `node` as a bitmask in shared memory (all threads of the block): a copy of the
+// prebuilt row for the root and for heavy nodes, else built from the child list.
+__device__ void build_mask(uint32_t* smask, const StepParams& p, int32_t node, int32_t cb, int32_t ce,
+                           int32_t* s_tmp) {
+    const uint32_t* src = nullptr;
     if (node == 0) {
-        for (int w = threadIdx.x; w < p.W; w += STEP_THREADS) smask[w] = __ldg(p.root_mask + w);
+        src = p.root_mask;
+    } else if (ce - cb > DISC_HEAVY_MIN) {
+        if (threadIdx.x == 0) *s_tmp = heavy_index(p.heavy_nodes, p.n_heavy, node);
+        __syncthreads();
+        const int32_t h = *s_tmp;
+        if (h >= 0) src = p.heavy_masks + size_t(h) * p.W;
+    }
+    if (src) {
+        for (int w = threadIdx.x; w < p.W; w += STEP_THREADS) smask[w] = __ldg(src + w);
     } else {
         for (int w = threadIdx.x; w < p.W; w += STEP_THREADS) smask[w] = 0u;
         __syncthreads();
@@ -205,17 +355,105 @@ __device__ int32_t warp_find_child(const int32_t* __restrict__ node_tok, int32_t
     return bal ? a + (__ffs(bal) - 1) : -1;
 }
 
-// ---- the kernel ---------------------------------------------------------------------------------
-template <int DT, bool VEC>
-__global__ void __launch_bounds__(STEP_THREADS, 4) disc_step_kernel(const StepParams p) {
+// ---- streaming loops ---------------------------------------------------------------------------
+// Bulk-copy ring: returns false if an mbarrier wait gave up.
+template <int DT, bool DENSE>
+__device__ bool stream_ring(Acc& a, const RowCtx& r, const char* rowp, int V, unsigned char* ring,
+                            uint64_t* full_bar, uint64_t* empty_bar, const uint32_t* smask) {
     using E = Elem<DT>;
-    constexpr int EPV = VEC ? E::EPV : 1;
-    extern __shared__ __align__(16) uint32_t smask[];
+    constexpr int EPV = E::EPV;
+    const int tid = threadIdx.x, lane = tid & 31;
+    const int nvec = V / EPV;
+    const uint32_t vec_bytes = uint32_t(nvec) * 16u;
+    const int n_chunks = int((vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
+    const uint32_t ring_s = smem_u32(ring);
+    bool ok = true;
+
+    auto issue = [&](int c) {
+        const int s = c % STAGES;
+        const uint32_t off = uint32_t(c) * CHUNK_BYTES;
+        const uint32_t bytes = min(uint32_t(CHUNK_BYTES), vec_bytes - off);
+        const uint32_t bar = smem_u32(&full_bar[s]);
+        mbar_expect_tx(bar, bytes);
+        bulk_g2s(ring_s + uint32_t(s) * CHUNK_BYTES, rowp + off, bytes, bar);
+    };
+    if (tid == 0) {
+        for (int c = 0; c < STAGES && c < n_chunks; ++c) issue(c);
+    }
+    for (int c = 0; c < n_chunks; ++c) {
+        const int s = c % STAGES;
+        const uint32_t use = uint32_t(c / STAGES);     // how often stage s was used before
+        // the give-up decision is taken per warp, so that all lanes leave the loop together
+        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&full_bar[s]), use & 1u))) { ok = false; break; }
+        uint4 raw[VPT];
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            const int in_chunk = j * STEP_THREADS + tid;
+            const int g = c * (CHUNK_BYTES / 16) + in_chunk;
+            if (g < nvec) raw[j] = *reinterpret_cast<const uint4*>(ring + s * CHUNK_BYTES + in_chunk * 16);
+        }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
+        // refill the stage released one iteration ago (every warp has long passed it)
+        if (tid == 0 && c >= 1 && c - 1 + STAGES < n_chunks) {
+            const int sp = (c - 1) % STAGES;
+            const uint32_t usep = uint32_t((c - 1) / STAGES);
+            if (!mbar_wait(smem_u32(&empty_bar[sp]), usep & 1u)) ok = false;
+            else issue(c - 1 + STAGES);
+        }
+        if (c == 0 && tid < nvec) {
+            float x[EPV];
+            E::unpack(raw[0], x);
+            float mx = x[0];
+#pragma unroll
+            for (int j = 1; j < EPV; ++j) mx = fmaxf(mx, x[j]);
+            set_reference(a, r, mx);
+            if constexpr (DENSE) update_bound(a, r);
+        }
+#pragma unroll
+        for (int j = 0; j < VPT; ++j) {
+            const int g = c * (CHUNK_BYTES / 16) + j * STEP_THREADS + tid;
+            if (g < nvec) {
+                float x[EPV];
+                E::unpack(raw[j], x);
+                consume<EPV, DENSE>(a, r, x, g * EPV, smask);
+            }
+        }
+    }
+    // ragged tail: V not a multiple of the vector width
+    const int v = nvec * EPV + tid;
+    if (v < V) {
+        float x[1] = {E::load(rowp, v)};
+        if (!a.touched) { set_reference(a, r, x[0]); if constexpr (DENSE) update_bound(a, r); }
+        consume<1, DENSE>(a, r, x, v, smask);
+    }
+    return ok;
+}
+
+template <int DT, bool DENSE>
+__device__ void stream_scalar(Acc& a, const RowCtx& r, const char* rowp, int V, const uint32_t* smask) {
+    using E = Elem<DT>;
+    for (int v = threadIdx.x; v < V; v += STEP_THREADS) {
+        float x[1] = {E::load(rowp, v)};
+        if (!a.touched) { set_reference(a, r, x[0]); if constexpr (DENSE) update_bound(a, r); }
+        consume<1, DENSE>(a, r, x, v, smask);
+    }
+}
+
+// ---- the kernel ---------------------------------------------------------------------------------
+template <int DT, bool RING>
+__global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepParams p) {
+    using E = Elem<DT>;
+    extern __shared__ __align__(128) unsigned char dyn_smem[];
+    unsigned char* ring = dyn_smem;                                             // RING_BYTES (RING only)
+    uint32_t* smask = reinterpret_cast<uint32_t*>(dyn_smem + (RING ? RING_BYTES : 0));
+    __shared__ __align__(8) uint64_t full_bar[STAGES];
+    __shared__ __align__(8) uint64_t empty_bar[STAGES];
     __shared__ float red_f[6][STEP_WARPS];
     __shared__ int32_t red_i[2][STEP_WARPS];
     __shared__ float scratch[STEP_WARPS];
     __shared__ float fin[4];        // (m, s) of the full row and of the valid set
-    __shared__ int32_t s_flag;
+    __shared__ int32_t s_flag, s_tmp, s_fault;
 
     const int64_t row = blockIdx.x;
     const int tid = threadIdx.x;
@@ -239,18 +477,32 @@ __global__ void __launch_bounds__(STEP_THREADS, 4) disc_step_kernel(const StepPa
         return;
     }
 
-    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
-    const RowRng rng{p.key, p.step, uint32_t(p.row_base + uint32_t(row))};
-    const bool dense = (c > GATHER_MAX) || (p.mask_out != nullptr);
-    float xref = E::load(rowp, 0);
-    if (!(fabsf(xref) < CUDART_INF_F)) xref = 0.f;
+    if (RING) {
+        if (tid == 0) {
+            for (int s = 0; s < STAGES; ++s) {
+                mbar_init(smem_u32(&full_bar[s]), 1);
+                mbar_init(smem_u32(&empty_bar[s]), STEP_WARPS);
+            }
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        }
+    }
+    if (tid == 0) s_fault = 0;
+    __syncthreads();
 
+    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
+    RowCtx r;
+    r.c2 = p.c2; r.inv_t = p.inv_t; r.key = p.key; r.step = p.step; r.row = uint32_t(p.row_base + uint32_t(row));
+    r.xref = E::load(rowp, 0);
+    if (!(fabsf(r.xref) < CUDART_INF_F)) r.xref = 0.f;
+    const bool dense = (c > DISC_HEAVY_MIN) || (p.mask_out != nullptr);
+
+    Acc a;
     MS ok{-CUDART_INF_F, 0.f};
-    Best best{-CUDART_INF_F, -1, -1};
     bool poisoned = false;
 
     if (dense) {
-        build_mask(smask, p, node, cb, ce);
+        build_mask(smask, p, node, cb, ce, &s_tmp);
         if (p.mask_out) {
             uint32_t* mo = p.mask_out + size_t(row) * p.W;
             for (int w = tid; w < p.W; w += STEP_THREADS) mo[w] = smask[w];
@@ -258,114 +510,44 @@ __global__ void __launch_bounds__(STEP_THREADS, 4) disc_step_kernel(const StepPa
     } else {
         // gather path: the few allowed logits are read directly
         for (int i = tid; i < c; i += STEP_THREADS) {
-            int32_t v = __ldg(p.node_tok + cb + i);
-            float x = E::load(rowp, v);
+            const int32_t v = __ldg(p.node_tok + cb + i);
+            const float x = E::load(rowp, v);
             // sum of 2^(x*c2) kept as 2^m * s; fma(x, c2, -m) is the exact product minus the
             // reference, so a large common offset of the logits costs no accuracy
             const float y = x * p.c2;
             if (!(y < CUDART_INF_F)) poisoned = true;                 // NaN or +inf: careful path
             else if (y > ok.m) { ok.s = ok.s * exp2f(ok.m - y) + exp2f(fmaf(x, p.c2, -y)); ok.m = y; }
             else if (y != -CUDART_INF_F) ok.s += exp2f(fmaf(x, p.c2, -ok.m));
-            uint4 r = philox4x32_10(uint32_t(v) >> 2, rng.step, rng.row, 0u, rng.key);
-            consider(best, gumbel_score(x, xref, p.inv_t, pick_word(r, v & 3)), v, cb + i);
+            const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, r.key);
+            const float score = gumbel_score(x, r.xref, r.inv_t, pick_word(w4, v & 3));
+            if (score > a.best.score) { a.best.score = score; a.best.tok = v; a.best.child = cb + i; }
         }
     }
 
     // ---- stream the row
-    const int nvec = p.V / EPV;
-    float mref = 0.f;
-    float s_all[2] = {0.f, 0.f};
-    float s_ok = 0.f;
-    bool touched = false;
-    bool lost = false;   // an allowed finite logit underflowed against this thread's reference
-
-    auto process = [&](const uint4& raw, float xs, int idx) {
-        float x[EPV];
-        if constexpr (VEC) E::unpack(raw, x); else x[0] = xs;
-        float e[EPV];
-#pragma unroll
-        for (int j = 0; j < EPV; ++j) {
-            e[j] = ex2_approx(fmaf(x[j], p.c2, -mref));
-            s_all[j & 1] += e[j];
-        }
-        if (dense) {
-            const int v0 = idx * EPV;
-            uint32_t bits = (smask[v0 >> 5] >> (v0 & 31)) & ((1u << EPV) - 1u);
-            if (bits) {
-#pragma unroll
-                for (int q = 0; q < (EPV + 3) / 4; ++q) {
-                    uint32_t nib = (bits >> (4 * q)) & 0xFu;
-                    if (nib) {
-                        uint4 r = philox4x32_10(uint32_t(v0 >> 2) + q, rng.step, rng.row, 0u, rng.key);
-#pragma unroll
-                        for (int l = 0; l < (EPV < 4 ? EPV : 4); ++l) {
-                            if ((nib >> l) & 1u) {
-                                const int j = 4 * q + l;
-                                const int v = v0 + j;
-                                s_ok += e[j];
-                                lost |= (e[j] == 0.f) && (x[j] > -CUDART_INF_F);
-                                consider(best, gumbel_score(x[j], xref, p.inv_t, pick_word(r, v & 3)), v, -1);
-                            }
-                        }
-                    }
-                }
-            }
-        }
-    };
-
-    if constexpr (VEC) {
-        const uint4* vp = reinterpret_cast<const uint4*>(rowp);
-        constexpr int STRIDE = STEP_THREADS * UNROLL;
-        for (int base = 0; base < nvec; base += STRIDE) {
-            uint4 raw[UNROLL];
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                int idx = base + u * STEP_THREADS + tid;
-                if (idx < nvec) raw[u] = ld_stream16(vp + idx);
-            }
-            if (base == 0 && tid < nvec) {
-                float x[EPV];
-                E::unpack(raw[0], x);
-                float mx = x[0];
-#pragma unroll
-                for (int j = 1; j < EPV; ++j) mx = fmaxf(mx, x[j]);
-                float r = mx * p.c2;
-                mref = (fabsf(r) < CUDART_INF_F) ? r : 0.f;
-                touched = true;
-            }
-#pragma unroll
-            for (int u = 0; u < UNROLL; ++u) {
-                int idx = base + u * STEP_THREADS + tid;
-                if (idx < nvec) process(raw[u], 0.f, idx);
-            }
-        }
-        // ragged tail: V not a multiple of the vector width
-        const int v = nvec * EPV + tid;
-        if (v < p.V) {
-            float x = E::load(rowp, v);
-            if (!touched) { float r = x * p.c2; mref = (fabsf(r) < CUDART_INF_F) ? r : 0.f; touched = true; }
-            float e = ex2_approx(fmaf(x, p.c2, -mref));
-            s_all[0] += e;
-            if (dense && ((smask[v >> 5] >> (v & 31)) & 1u)) {
-                s_ok += e;
-                lost |= (e == 0.f) && (x > -CUDART_INF_F);
-                uint4 r = philox4x32_10(uint32_t(v) >> 2, rng.step, rng.row, 0u, rng.key);
-                consider(best, gumbel_score(x, xref, p.inv_t, pick_word(r, v & 3)), v, -1);
-            }
-        }
+    bool waits_ok = true;
+    if (RING) {
+        waits_ok = dense ? stream_ring<DT, true>(a, r, rowp, p.V, ring, full_bar, empty_bar, smask)
+                         : stream_ring<DT, false>(a, r, rowp, p.V, ring, full_bar, empty_bar, smask);
     } else {
-        for (int idx = tid; idx < p.V; idx += STEP_THREADS) {
-            float x = E::load(rowp, idx);
-            if (!touched) { float r = x * p.c2; mref = (fabsf(r) < CUDART_INF_F) ? r : 0.f; touched = true; }
-            process(uint4{}, x, idx);
-        }
+        if (dense) stream_scalar<DT, true>(a, r, rowp, p.V, smask);
+        else stream_scalar<DT, false>(a, r, rowp, p.V, smask);
     }
+    if (!waits_ok) s_fault = 1;
 
-    MS all = touched ? MS{mref, s_all[0] + s_all[1]} : MS{-CUDART_INF_F, 0.f};
-    if (dense) ok = touched ? MS{mref, s_ok} : MS{-CUDART_INF_F, 0.f};
+    MS all = a.touched ? MS{a.mref, a.s_all0 + a.s_all1} : MS{-CUDART_INF_F, 0.f};
+    if (dense) ok = a.touched ? MS{a.mref, a.s_ok} : MS{-CUDART_INF_F, 0.f};
     if (poisoned) ok.s = CUDART_NAN_F;
+    Best best = a.best;
 
-    const int any_lost = __syncthreads_or(lost ? 1 : 0);
+    const int any_lost = __syncthreads_or(a.lost ? 1 : 0);
+    if (s_fault) {
+        // A bulk copy never signalled completion.  Report it and leave the row untouched; give
+        // outstanding copies a bounded time to land before the block's shared memory is released.
+        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_FAULT; }
+        return;
+    }
 
     // ---- block reduction of (all, ok, best)
 #pragma unroll
@@ -403,27 +585,37 @@ __global__ void __launch_bounds__(STEP_THREADS, 4) disc_step_kernel(const StepPa
             ok = ms_merge(ok, k2);
             best = best_merge(best, b2);
         }
-        if (lane == 0) {
-            fin[0] = all.m; fin[1] = all.s; fin[2] = ok.m; fin[3] = ok.s;
-            const float l2_all = all.m + log2f(all.s);
-            const float l2_ok = ok.m + log2f(ok.s);
-            // the fast sums are trusted only when both are finite and no allowed term was lost
-            s_flag = (fabsf(l2_all) < CUDART_INF_F && fabsf(l2_ok) < CUDART_INF_F && !any_lost) ? 0 : 1;
-        }
+    }
+    __syncthreads();       // every warp has read its red_* partials; lane 0 may now overwrite slot 0
+    if (warp == 0 && lane == 0) {
+        fin[0] = all.m; fin[1] = all.s; fin[2] = ok.m; fin[3] = ok.s;
+        const float l2_all = all.m + log2f(all.s);
+        const float l2_ok = ok.m + log2f(ok.s);
+        // the fast sums are trusted only when both are finite and no allowed term was lost
+        s_flag = (fabsf(l2_all) < CUDART_INF_F && fabsf(l2_ok) < CUDART_INF_F && !any_lost) ? 0 : 1;
+        red_f[4][0] = best.score; red_i[0][0] = best.tok; red_i[1][0] = best.child;
     }
     __syncthreads();
 
     if (s_flag) {
         // ---- careful path: plain two-pass log-sum-exp over the row with an explicit mask and
-        // separate maxima for the full row and for the valid set
-        if (!dense) build_mask(smask, p, node, cb, ce);
+        // separate maxima for the full row and for the valid set; in the dense path the scores of
+        // all allowed tokens are evaluated exactly again (its skip bound relies on terms that did
+        // not underflow)
+        if (!dense) build_mask(smask, p, node, cb, ce, &s_tmp);
         float mx_all = -CUDART_INF_F, mx_ok = -CUDART_INF_F;
         int nan_all = 0, nan_ok = 0;
+        Best cbest{-CUDART_INF_F, -1, -1};
         for (int v = tid; v < p.V; v += STEP_THREADS) {
             const float x = E::load(rowp, v);
             const bool allowed = (smask[v >> 5] >> (v & 31)) & 1u;
             if (x != x) { nan_all = 1; nan_ok |= allowed; }
             else { mx_all = fmaxf(mx_all, x); if (allowed) mx_ok = fmaxf(mx_ok, x); }
+            if (allowed && dense) {
+                const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, r.key);
+                const float score = gumbel_score(x, r.xref, r.inv_t, pick_word(w4, v & 3));
+                if (score > cbest.score) { cbest.score = score; cbest.tok = v; }
+            }
         }
         mx_all = block_max(mx_all, scratch);
         mx_ok = block_max(mx_ok, scratch);
@@ -440,6 +632,21 @@ __global__ void __launch_bounds__(STEP_THREADS, 4) disc_step_kernel(const StepPa
         }
         sum_all = block_sum(sum_all, scratch);
         sum_ok = block_sum(sum_ok, scratch);
+        if (dense) {
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                Best b2{__shfl_xor_sync(0xffffffffu, cbest.score, o), __shfl_xor_sync(0xffffffffu, cbest.tok, o), -1};
+                cbest = best_merge(cbest, b2);
+            }
+            __syncthreads();
+            if (lane == 0) { red_f[5][warp] = cbest.score; red_i[0][warp] = cbest.tok; }
+            __syncthreads();
+            if (tid == 0) {
+                Best b{red_f[5][0], red_i[0][0], -1};
+                for (int w = 1; w < STEP_WARPS; ++w) b = best_merge(b, Best{red_f[5][w], red_i[0][w], -1});
+                red_f[4][0] = b.score; red_i[0][0] = b.tok; red_i[1][0] = -1;
+            }
+        }
         if (tid == 0) {
             // (m, s) with value 2^m * s; +inf maximum -> (+inf, 1), empty or all -inf -> (-inf, 0)
             fin[0] = nan_all ? CUDART_NAN_F : (fin_all ? r_all : mx_all);
@@ -452,10 +659,7 @@ __global__ void __launch_bounds__(STEP_THREADS, 4) disc_step_kernel(const StepPa
 
     // ---- finalise: one warp moves the row's cursor to the chosen child
     if (warp == 0) {
-        best.score = __shfl_sync(0xffffffffu, best.score, 0);
-        best.tok = __shfl_sync(0xffffffffu, best.tok, 0);
-        best.child = __shfl_sync(0xffffffffu, best.child, 0);
-        int32_t tok = best.tok, child = best.child;
+        int32_t tok = red_i[0][0], child = red_i[1][0];
         if (tok < 0) { tok = __ldg(p.node_tok + cb); child = cb; }     // no finite score: lowest id
         if (child < 0) {
             child = (node == 0) ? __ldg(p.root_child + tok) : warp_find_child(p.node_tok, cb, ce, tok);
@@ -509,13 +713,11 @@ __global__ void k_sampling_uniforms(PhiloxKey key, uint32_t step, uint32_t row, 
     out[i] = uniform_from_bits(pick_word(r, v & 3));
 }
 
-template <int DT, bool VEC>
+template <int DT, bool RING>
 int launch_step(const StepParams& p, int64_t n, size_t smem, cudaStream_t st) {
-    if (smem > 48 * 1024) {
-        DISC_CUDA(cudaFuncSetAttribute(disc_step_kernel<DT, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       int(smem)));
-    }
-    disc_step_kernel<DT, VEC><<<unsigned(n), STEP_THREADS, smem, st>>>(p);
+    DISC_CUDA(cudaFuncSetAttribute(disc_step_kernel<DT, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                   int(smem)));
+    disc_step_kernel<DT, RING><<<unsigned(n), STEP_THREADS, smem, st>>>(p);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }
@@ -546,8 +748,8 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     if (ld < s->V || row_base < 0 || (seq_tokens && seq_ld <= 0)) return DISC_ERR_ARG;
     if (!(inv_temperature > 0.f) || !(inv_temperature <= 3.0e38f)) return DISC_ERR_ARG;
     if (dtype != DISC_F32 && dtype != DISC_BF16) return DISC_ERR_UNSUPPORTED;
-    const size_t smem = (size_t(s->W) * 4 + 15) & ~size_t(15);
-    if (smem > 200 * 1024) return DISC_ERR_UNSUPPORTED;
+    const size_t mask_bytes = (size_t(s->W) * 4 + 15) & ~size_t(15);
+    if (mask_bytes > 160 * 1024) return DISC_ERR_UNSUPPORTED;
 
     StepParams p;
     p.logits = logits; p.ld = ld; p.inv_t = inv_temperature; p.c2 = inv_temperature * LOG2E_F;
@@ -556,13 +758,17 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     p.token_out = token_out; p.seq_tokens = seq_tokens; p.seq_ld = seq_ld;
     p.logq_out = logq_out; p.logp_out = logp_out; p.mask_out = mask_out; p.status_out = status_out;
     p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
-    p.root_child = s->root_child; p.root_mask = s->root_mask; p.V = s->V; p.W = s->W; p.M = s->M;
+    p.root_child = s->root_child; p.root_mask = s->root_mask;
+    p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
+    p.V = s->V; p.W = s->W; p.M = s->M;
 
     const size_t esize = dtype == DISC_F32 ? 4 : 2;
-    const bool vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
+    // the bulk-copy ring needs 16-byte aligned rows; other layouts take the scalar path
+    const bool ring = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
+    const size_t smem = mask_bytes + (ring ? RING_BYTES : 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dtype == DISC_F32) return vec ? launch_step<DISC_F32, true>(p, n, smem, st) : launch_step<DISC_F32, false>(p, n, smem, st);
-    return vec ? launch_step<DISC_BF16, true>(p, n, smem, st) : launch_step<DISC_BF16, false>(p, n, smem, st);
+    if (dtype == DISC_F32) return ring ? launch_step<DISC_F32, true>(p, n, smem, st) : launch_step<DISC_F32, false>(p, n, smem, st);
+    return ring ? launch_step<DISC_BF16, true>(p, n, smem, st) : launch_step<DISC_BF16, false>(p, n, smem, st);
 }
 
 int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t v0, int32_t n, float* out,
