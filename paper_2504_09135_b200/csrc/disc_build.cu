@@ -225,6 +225,7 @@ int build_impl(const int32_t* tokens, const int64_t* row_offsets, int64_t n, int
     DISC_CUDA(cudaGetDevice(&S->device));
     S->V = V;
     S->W = (V + 31) / 32;
+    S->Wp = (S->W + 3) & ~3;
 
     DevBuf in_tok, in_off64, in_off, len, err, lmax_d;
     DISC_CUDA(in_tok.alloc(size_t(E_in) * 4));
@@ -353,7 +354,7 @@ int build_impl(const int32_t* tokens, const int64_t* row_offsets, int64_t n, int
     DISC_CUDA(node_tok.alloc(size_t(M) * 4));
     DISC_CUDA(node_lo.alloc(size_t(M) * 4));
     DISC_CUDA(child_begin.alloc(size_t(M + 1) * 4));
-    DISC_CUDA(root_mask.alloc(size_t(S->W) * 4));
+    DISC_CUDA(root_mask.alloc(size_t(S->Wp) * 4));
     DISC_CUDA(root_child.alloc(size_t(V) * 4));
     bool have_next = false;
     for (int32_t d = l_max - 1; d >= 0; --d) {
@@ -379,7 +380,7 @@ int build_impl(const int32_t* tokens, const int64_t* row_offsets, int64_t n, int
         DISC_CUDA(cudaMemcpyAsync(child_begin.as<int32_t>() + M, &sentinel, 4, cudaMemcpyHostToDevice, st));
         DISC_CUDA(cudaStreamSynchronize(st));
     }
-    DISC_CUDA(cudaMemsetAsync(root_mask.p, 0, size_t(S->W) * 4, st));
+    DISC_CUDA(cudaMemsetAsync(root_mask.p, 0, size_t(S->Wp) * 4, st));
     k_fill_i32<<<blocks_for(V), TPB, 0, st>>>(root_child.as<int32_t>(), -1, V);
     k_root_tables<<<blocks_for(level_n[0]), TPB, 0, st>>>(node_tok.as<int32_t>(), 1, level_n[0],
                                                          root_child.as<int32_t>(), root_mask.as<uint32_t>());
@@ -405,11 +406,11 @@ int build_impl(const int32_t* tokens, const int64_t* row_offsets, int64_t n, int
         DISC_CUDA(cudaMemcpyAsync(&H, n_sel.p, 4, cudaMemcpyDeviceToHost, st));
         DISC_CUDA(cudaStreamSynchronize(st));
         S->n_heavy = H;
-        DISC_CUDA(heavy_masks.alloc(size_t(H > 0 ? H : 1) * size_t(S->W) * 4));
+        DISC_CUDA(heavy_masks.alloc(size_t(H > 0 ? H : 1) * size_t(S->Wp) * 4));
         if (H > 0) {
-            DISC_CUDA(cudaMemsetAsync(heavy_masks.p, 0, size_t(H) * size_t(S->W) * 4, st));
+            DISC_CUDA(cudaMemsetAsync(heavy_masks.p, 0, size_t(H) * size_t(S->Wp) * 4, st));
             k_heavy_masks<<<unsigned(H), 256, 0, st>>>(heavy_nodes.as<int32_t>(), child_begin.as<int32_t>(),
-                                                     node_tok.as<int32_t>(), S->W, heavy_masks.as<uint32_t>());
+                                                     node_tok.as<int32_t>(), S->Wp, heavy_masks.as<uint32_t>());
             DISC_CUDA(cudaGetLastError());
             DISC_CUDA(cudaStreamSynchronize(st));
         }

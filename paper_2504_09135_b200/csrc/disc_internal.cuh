@@ -9,6 +9,7 @@
 struct disc_set {
     int32_t V = 0;            // vocabulary size
     int32_t W = 0;            // mask words per row
+    int32_t Wp = 0;           // row stride of the prebuilt masks in words (W rounded up to 4: 16-byte rows)
     int32_t l_max = 0;
     int64_t N = 0;            // members
     int64_t E = 0;            // table entries
@@ -91,6 +92,40 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
         c2 = n2;
         k0 += 0x9E3779B9u;
         k1 += 0xBB67AE85u;
+    }
+    return make_uint4(c0, c1, c2, c3);
+}
+
+// The ten round keys (k0 + r*W0, k1 + r*W1), computed once on the host and passed as kernel
+// parameters, so that a round is two wide multiplies and two three-input XORs.
+struct PhiloxRoundKeys {
+    uint32_t k[20];
+};
+
+inline PhiloxRoundKeys philox_round_keys(uint64_t seed) {
+    PhiloxRoundKeys rk;
+    uint32_t k0 = uint32_t(seed), k1 = uint32_t(seed >> 32);
+    for (int r = 0; r < 10; ++r) {
+        rk.k[2 * r] = k0;
+        rk.k[2 * r + 1] = k1;
+        k0 += 0x9E3779B9u;
+        k1 += 0xBB67AE85u;
+    }
+    return rk;
+}
+
+__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                               const PhiloxRoundKeys& rk) {
+#pragma unroll
+    for (int r = 0; r < 10; ++r) {
+        uint64_t p0 = uint64_t(0xD2511F53u) * c0;
+        uint64_t p1 = uint64_t(0xCD9E8D57u) * c2;
+        uint32_t n0 = uint32_t(p1 >> 32) ^ c1 ^ rk.k[2 * r];
+        uint32_t n2 = uint32_t(p0 >> 32) ^ c3 ^ rk.k[2 * r + 1];
+        c1 = uint32_t(p1);
+        c3 = uint32_t(p0);
+        c0 = n0;
+        c2 = n2;
     }
     return make_uint4(c0, c1, c2, c3);
 }

@@ -24,7 +24,7 @@ struct MaskParams {
     uint8_t* status_out;
     const int32_t *node_tok, *node_lo, *child_begin, *root_child, *heavy_nodes;
     const uint32_t *root_mask, *heavy_masks;
-    int32_t V, W, N, n_heavy;
+    int32_t V, W, Wp, N, n_heavy;
 };
 
 __device__ __forceinline__ int32_t find_child(const int32_t* __restrict__ node_tok, int32_t cb, int32_t ce, int32_t t,
@@ -90,7 +90,7 @@ __global__ void __launch_bounds__(MASK_THREADS) disc_mask_kernel(const MaskParam
         if (ok && node == 0) src = p.root_mask;
         else if (ok && ce - cb > DISC_HEAVY_MIN) {
             const int32_t h = disc::heavy_index(p.heavy_nodes, p.n_heavy, node);
-            if (h >= 0) src = p.heavy_masks + size_t(h) * p.W;
+            if (h >= 0) src = p.heavy_masks + size_t(h) * p.Wp;
         }
         uint32_t* row = p.mask_out + size_t(i) * p.W;
         if (VEC) {
@@ -137,7 +137,7 @@ extern "C" int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t pre
     p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
     p.root_child = s->root_child; p.root_mask = s->root_mask;
     p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
-    p.V = s->V; p.W = s->W; p.N = int32_t(s->N);
+    p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.N = int32_t(s->N);
 
     int dev = 0, sms = 0;
     DISC_CUDA(cudaGetDevice(&dev));

@@ -5,28 +5,38 @@
 // One thread block per row.
 //   * Streaming.  The row's logits are pulled into a shared-memory ring by bulk asynchronous
 //     copies (cp.async.bulk + mbarrier, one elected thread issues them), so several chunks are in
-//     flight per block whatever the register budget; rows that are not 16-byte aligned take a
-//     plain scalar-load path.
+//     flight per block whatever the register budget.  The first chunks are issued before the
+//     block reads the prefix index.  Rows that are not 16-byte aligned take a scalar-load path.
 //   * Sums.  Each thread accumulates sum 2^(x*c - ref) against its own reference (the maximum of
-//     the first vector it sees), c = log2(e)/T: one FMA, one ex2 and one add per logit.  Partial
-//     sums are kept as (m, s) pairs meaning 2^m * s and merged exactly.  All differences are formed
-//     between references before any large value is added, so a common offset of the logits does
-//     not cost accuracy.
+//     the first vector it sees), c = log2(e)/T.  Per pair of logits: two unpack operations, one
+//     packed fp32x2 FMA, two ex2 and one packed add.  Partial sums are kept as (m, s) pairs meaning
+//     2^m * s and merged exactly.  All differences are formed between references before any large
+//     value is added, so a common offset of the logits does not cost accuracy.
 //   * Valid set.  The prefix index gives the row's children as a contiguous list.  Rows with at
 //     most DISC_HEAVY_MIN children gather their few logits directly ("gather path").  Rows with
-//     more use a bitmask in shared memory (prebuilt at set-build time) that the streaming loop
-//     consults ("dense path").
+//     more have a prebuilt bitmask row in global memory; its slice travels into the ring stage next
+//     to the logits it covers ("dense path").
 //   * Sampling.  token = argmax over allowed v of (x_v - xref)/T + g_v with g_v = -log(-log u_v),
 //     u_v from Philox4x32-10 keyed by (token, step, row).  In the dense path a token is evaluated
 //     exactly only if it can still win: with w = 1 - u, g > t implies w < e^-t, so a token whose
 //     w is at least e^(z - best) (times a safety factor) is skipped without taking a logarithm;
-//     e^(z - best) is the already computed 2^(x*c - ref) times a per-thread constant.
-//   * A row whose fast sums are not finite, or that lost an allowed term to underflow, is redone
-//     by a plain two-pass routine with exact scores ("careful path").
+//     e^(z - best) is the already computed 2^(x*c - ref) times a per-thread constant.  `best` is the
+//     best score any lane of the warp has seen (shared once per chunk), which keeps the number of
+//     exact evaluations per warp near log(tokens).
+//   * A row whose fast sums are not finite, or whose valid mass is so small that terms may have
+//     underflowed against a thread's reference, is redone by a plain two-pass routine with exact
+//     scores ("careful path").
 
 #include <math_constants.h>
 
 #include "disc_internal.cuh"
+
+#ifndef DISC_STAGES
+#define DISC_STAGES 3
+#endif
+#ifndef DISC_MIN_BLOCKS
+#define DISC_MIN_BLOCKS 4
+#endif
 
 namespace {
 
@@ -34,22 +44,26 @@ using namespace disc;
 
 constexpr int STEP_THREADS = 256;
 constexpr int STEP_WARPS = STEP_THREADS / 32;
-constexpr int CHUNK_BYTES = 8192;                       // one ring stage
-constexpr int STAGES = 4;
-constexpr int VPT = CHUNK_BYTES / 16 / STEP_THREADS;    // 16-byte vectors per thread and stage
-constexpr int RING_BYTES = CHUNK_BYTES * STAGES;
+constexpr int VPT = 4;                                   // 16-byte vectors per thread and stage
+constexpr int CHUNK_VECS = VPT * STEP_THREADS;
+constexpr int CHUNK_BYTES = CHUNK_VECS * 16;             // logits of one ring stage: 16 KB
+constexpr int MASK_SLICE_MAX = CHUNK_VECS;               // mask bytes of one stage (bf16: 8 tokens per vector)
+constexpr int STAGE_BYTES = CHUNK_BYTES + MASK_SLICE_MAX;
+constexpr int STAGES = DISC_STAGES;
+constexpr int RING_BYTES = STAGE_BYTES * STAGES;
 constexpr uint64_t WAIT_LIMIT_NS = 250ull * 1000 * 1000;  // an mbarrier wait gives up after 0.25 s
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
 constexpr float SAFETY = 1.0009765625f;                 // 1 + 2^-10 on the skip bound
 constexpr float TWO_M24 = 5.9604644775390625e-08f;      // 2^-24: smallest possible w
+constexpr float MASS_FLOOR_LOG2 = 60.f;   // dense sums are trusted while log2(mass) >= -60 (see below)
 
 struct StepParams {
     const void* logits;
     int64_t ld;
     float inv_t;
     float c2;            // inv_t * log2(e)
-    PhiloxKey key;
+    PhiloxRoundKeys rk;
     uint32_t step;
     uint32_t row_base;
     // state
@@ -66,7 +80,7 @@ struct StepParams {
     // set
     const int32_t *node_tok, *node_lo, *child_begin, *root_child, *heavy_nodes;
     const uint32_t *root_mask, *heavy_masks;
-    int32_t V, W, n_heavy;
+    int32_t V, W, Wp, n_heavy;
     int64_t M;
 };
 
@@ -144,18 +158,19 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t
                  : "memory");
 }
 
+// ---- element types ------------------------------------------------------------------------------
 template <int DT>
 struct Elem;
 template <>
 struct Elem<DISC_F32> {
     static constexpr int SIZE = 4;
-    static constexpr int EPV = 4;
+    static constexpr int EPV = 4;       // elements per 16-byte vector
     __device__ static __forceinline__ float load(const void* base, int64_t i) {
         return __ldg(static_cast<const float*>(base) + i);
     }
-    __device__ static __forceinline__ void unpack(const uint4& v, float (&x)[4]) {
-        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
-        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&x)[2]) {
+        x[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
+        x[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
     }
 };
 template <>
@@ -165,18 +180,20 @@ struct Elem<DISC_BF16> {
     __device__ static __forceinline__ float load(const void* base, int64_t i) {
         return __uint_as_float(uint32_t(__ldg(static_cast<const unsigned short*>(base) + i)) << 16);
     }
-    __device__ static __forceinline__ void unpack(const uint4& v, float (&x)[8]) {
-        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xffff0000u);
-        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xffff0000u);
-        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xffff0000u);
-        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xffff0000u);
+    __device__ static __forceinline__ float2 pair(uint32_t w) {
+        return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    }
+    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&x)[4]) {
+        x[0] = pair(v.x); x[1] = pair(v.y); x[2] = pair(v.z); x[3] = pair(v.w);
     }
 };
 
 // Gumbel-perturbed score of a token with raw logit x, relative to the row's reference logit xref.
 // The argmax does not depend on the common shift, and subtracting before scaling keeps the score
-// accurate to a few ulp of (x - xref) whatever offset the logits carry.
-__device__ __forceinline__ float gumbel_score(float x, float xref, float inv_t, uint32_t word) {
+// accurate to a few ulp of (x - xref) whatever offset the logits carry.  Kept out of line: it is
+// reached for a handful of tokens per warp and row, and inlining it at every call site would
+// multiply the size of the streaming loop.
+__device__ __noinline__ float gumbel_score(float x, float xref, float inv_t, uint32_t word) {
     return (x - xref) * inv_t + gumbel_from_uniform(uniform_from_bits(word));
 }
 
@@ -186,33 +203,38 @@ __device__ __forceinline__ float complement_uniform(uint32_t word) {
     return __uint_as_float(0x3f800000u | ((~word) >> 9)) - 0.99999994039535522f;
 }
 
+__device__ __forceinline__ bool mask_bit(const uint32_t* __restrict__ gmask, int v) {
+    return (__ldg(gmask + (v >> 5)) >> (v & 31)) & 1u;
+}
+
 // Per-thread accumulators of the streaming loop.
 struct Acc {
     float mref = 0.f;        // reference exponent (log2 domain) of this thread's sums
-    float s_all0 = 0.f, s_all1 = 0.f;
-    float s_ok = 0.f;
+    float2 sa = {0.f, 0.f}, sb = {0.f, 0.f};      // four partial sums over all logits
+    float2 ok2 = {0.f, 0.f};                      // two partial sums over the allowed logits
     bool touched = false;
-    bool lost = false;       // an allowed term underflowed to zero against mref
     // sampling
     Best best{-__builtin_huge_valf(), -1, -1};
-    float cbound = __builtin_huge_valf();   // SAFETY * 2^(mref - xref*c - best*log2e): e * cbound bounds e^(z - best)
+    float bound_best = -__builtin_huge_valf();   // best score known to this warp (>= best.score)
+    float cbase = 0.f;                            // mref - xref*c
+    float cbound = __builtin_huge_valf();   // SAFETY * 2^(cbase - bound_best*log2e): e*cbound >= e^(z-best)
 };
 
 struct RowCtx {
     float c2, inv_t, xref;
-    PhiloxKey key;
     uint32_t step, row;
 };
+
+__device__ __forceinline__ void update_bound(Acc& a) {
+    a.cbound = SAFETY * exp2f(a.cbase - a.bound_best * LOG2E_F);
+}
 
 __device__ __forceinline__ void set_reference(Acc& a, const RowCtx& r, float xmax) {
     const float m = xmax * r.c2;
     a.mref = (fabsf(m) < CUDART_INF_F) ? m : 0.f;
+    a.cbase = fmaf(-r.xref, r.c2, a.mref);      // one rounding of the exact difference
     a.touched = true;
-}
-
-__device__ __forceinline__ void update_bound(Acc& a, const RowCtx& r) {
-    // exponent of e^(z - best) / 2^(x*c - mref); fma keeps (mref - xref*c) exact to one rounding
-    a.cbound = SAFETY * exp2f(fmaf(-r.xref, r.c2, a.mref) - a.best.score * LOG2E_F);
+    update_bound(a);
 }
 
 __device__ __forceinline__ void exact_candidate(Acc& a, const RowCtx& r, float x, uint32_t word, int32_t v) {
@@ -220,58 +242,103 @@ __device__ __forceinline__ void exact_candidate(Acc& a, const RowCtx& r, float x
     // tie.  NaN and -inf scores never win; a row without any finite score falls back to its
     // lowest valid token at the end.
     const float score = gumbel_score(x, r.xref, r.inv_t, word);
-    if (score > a.best.score) {
-        a.best.score = score; a.best.tok = v; a.best.child = -1;
-        update_bound(a, r);
+    if (score > a.best.score) { a.best.score = score; a.best.tok = v; a.best.child = -1; }
+    if (score > a.bound_best) { a.bound_best = score; update_bound(a); }
+}
+
+// share the best score of the warp's lanes (called at warp-uniform points)
+__device__ __forceinline__ void share_bound(Acc& a) {
+    float b = a.bound_best;
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) b = fmaxf(b, __shfl_xor_sync(0xffffffffu, b, o));
+    a.bound_best = b;
+    update_bound(a);
+}
+
+// the four tokens 4g .. 4g+3 of one Philox counter; nib = which of them are allowed
+__device__ __forceinline__ void sample_group(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, uint32_t g,
+                                             uint32_t nib, float x0, float x1, float x2, float x3, float e0,
+                                             float e1, float e2, float e3) {
+    // No token of this group can win if even the largest noise is not enough: w >= 2^-24 always,
+    // so e*cbound < 2^-24 for all four means "skip" without drawing the random numbers.
+#ifdef DISC_EXP_NOSAMPLE
+    return;
+#endif
+    const float emax = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
+    if (emax * a.cbound < TWO_M24) return;
+#ifdef DISC_EXP_CHEAPRNG
+    const uint32_t hh = (g * 2654435761u) ^ (r.row * 40503u) ^ rk.k[0];
+    const uint4 w4 = make_uint4(hh, hh * 3u, hh * 5u, hh * 7u);
+#else
+    const uint4 w4 = philox4x32_10(g, r.step, r.row, 0u, rk);
+#endif
+    const int32_t v = int32_t(g << 2);
+    if ((nib & 1u) && !(complement_uniform(w4.x) >= e0 * a.cbound)) exact_candidate(a, r, x0, w4.x, v);
+    if ((nib & 2u) && !(complement_uniform(w4.y) >= e1 * a.cbound)) exact_candidate(a, r, x1, w4.y, v + 1);
+    if ((nib & 4u) && !(complement_uniform(w4.z) >= e2 * a.cbound)) exact_candidate(a, r, x2, w4.z, v + 2);
+    if ((nib & 8u) && !(complement_uniform(w4.w) >= e3 * a.cbound)) exact_candidate(a, r, x3, w4.w, v + 3);
+}
+
+// one 16-byte vector of logits starting at token v0 (a multiple of the vector width);
+// bits = allowed flags of its EPV tokens (dense path only)
+template <int DT, bool DENSE>
+__device__ __forceinline__ void consume_vec(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const uint4& raw,
+                                            int v0, uint32_t bits) {
+    using E = Elem<DT>;
+    constexpr int NP = E::EPV / 2;
+    float2 x[NP], e[NP];
+    E::unpack(raw, x);
+    const float2 cc = make_float2(r.c2, r.c2), nm = make_float2(-a.mref, -a.mref);
+#pragma unroll
+    for (int i = 0; i < NP; ++i) {
+        const float2 y = __ffma2_rn(x[i], cc, nm);
+        e[i] = make_float2(ex2_approx(y.x), ex2_approx(y.y));
+    }
+    if constexpr (!DENSE) {
+#pragma unroll
+        for (int i = 0; i < NP; i += 2) {
+            a.sa = __fadd2_rn(a.sa, e[i]);
+            a.sb = __fadd2_rn(a.sb, e[i + 1]);
+        }
+    } else {
+        float2 t = __fadd2_rn(e[0], e[1]);
+        if constexpr (NP == 4) t = __fadd2_rn(t, __fadd2_rn(e[2], e[3]));
+        a.sa = __fadd2_rn(a.sa, t);
+        constexpr uint32_t FULL = (1u << E::EPV) - 1u;
+        if (bits) {
+            if (bits == FULL) {
+                a.ok2 = __fadd2_rn(a.ok2, t);
+            } else {
+#pragma unroll
+                for (int i = 0; i < NP; ++i) {
+                    a.ok2.x += ((bits >> (2 * i)) & 1u) ? e[i].x : 0.f;
+                    a.ok2.y += ((bits >> (2 * i + 1)) & 1u) ? e[i].y : 0.f;
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < NP / 2; ++q) {
+                const uint32_t nib = (bits >> (4 * q)) & 0xFu;
+                if (nib)
+                    sample_group(a, r, rk, uint32_t(v0 >> 2) + q, nib, x[2 * q].x, x[2 * q].y, x[2 * q + 1].x,
+                                 x[2 * q + 1].y, e[2 * q].x, e[2 * q].y, e[2 * q + 1].x, e[2 * q + 1].y);
+            }
+        }
     }
 }
 
-// one vector of EPV logits starting at token v0
-template <int EPV, bool DENSE>
-__device__ __forceinline__ void consume(Acc& a, const RowCtx& r, const float (&x)[EPV], int v0,
-                                        const uint32_t* __restrict__ smask) {
-    float e[EPV];
-#pragma unroll
-    for (int j = 0; j < EPV; ++j) e[j] = ex2_approx(fmaf(x[j], r.c2, -a.mref));
-#pragma unroll
-    for (int j = 0; j < EPV; j += 2) {
-        a.s_all0 += e[j];
-        if (j + 1 < EPV) a.s_all1 += e[j + 1];
-    }
-    if constexpr (DENSE) {
-        const uint32_t bits = (smask[v0 >> 5] >> (v0 & 31)) & ((1u << EPV) - 1u);
-        if (bits) {
-#pragma unroll
-            for (int j = 0; j < EPV; ++j) {
-                const bool on = (bits >> j) & 1u;
-                a.s_ok += on ? e[j] : 0.f;
-                a.lost |= on && !(e[j] > 0.f);
-            }
-#pragma unroll
-            for (int q = 0; q < (EPV + 3) / 4; ++q) {
-                const uint32_t nib = (bits >> (4 * q)) & 0xFu;
-                if (nib) {
-                    // no token of this group can win if even the largest noise is not enough:
-                    // w >= 2^-24 always, so e*cbound < 2^-24 for all four means "skip" without
-                    // drawing the random numbers
-                    float emax = e[4 * q];
-#pragma unroll
-                    for (int l = 1; l < (EPV < 4 ? EPV : 4); ++l) emax = fmaxf(emax, e[4 * q + l]);
-                    if (!(emax * a.cbound < TWO_M24)) {
-                        const uint4 w4 = philox4x32_10(uint32_t(v0 >> 2) + q, r.step, r.row, 0u, r.key);
-#pragma unroll
-                        for (int l = 0; l < (EPV < 4 ? EPV : 4); ++l) {
-                            if ((nib >> l) & 1u) {
-                                const int j = 4 * q + l;
-                                const int v = v0 + j;
-                                const uint32_t word = pick_word(w4, v & 3);
-                                if (!(complement_uniform(word) >= e[j] * a.cbound))
-                                    exact_candidate(a, r, x[j], word, v);
-                            }
-                        }
-                    }
-                }
-            }
+// one logit (scalar path and ragged tail); the allowed flag comes from the global mask row
+template <bool DENSE>
+__device__ __forceinline__ void consume_one(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, float x, int v,
+                                            const uint32_t* __restrict__ gmask) {
+    if (!a.touched) set_reference(a, r, x);
+    const float e = ex2_approx(fmaf(x, r.c2, -a.mref));
+    a.sa.x += e;
+    if (DENSE && mask_bit(gmask, v)) {
+        a.ok2.x += e;
+        if (!(e * a.cbound < TWO_M24)) {
+            const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, rk);
+            const uint32_t word = pick_word(w4, v & 3);
+            if (!(complement_uniform(word) >= e * a.cbound)) exact_candidate(a, r, x, word, v);
         }
     }
 }
@@ -308,32 +375,6 @@ __device__ float block_sum(float v, float* scratch) {
     return r;
 }
 
-// Valid set of `node` as a bitmask in shared memory (all threads of the block): a copy of the
-// prebuilt row for the root and for heavy nodes, else built from the child list.
-__device__ void build_mask(uint32_t* smask, const StepParams& p, int32_t node, int32_t cb, int32_t ce,
-                           int32_t* s_tmp) {
-    const uint32_t* src = nullptr;
-    if (node == 0) {
-        src = p.root_mask;
-    } else if (ce - cb > DISC_HEAVY_MIN) {
-        if (threadIdx.x == 0) *s_tmp = heavy_index(p.heavy_nodes, p.n_heavy, node);
-        __syncthreads();
-        const int32_t h = *s_tmp;
-        if (h >= 0) src = p.heavy_masks + size_t(h) * p.W;
-    }
-    if (src) {
-        for (int w = threadIdx.x; w < p.W; w += STEP_THREADS) smask[w] = __ldg(src + w);
-    } else {
-        for (int w = threadIdx.x; w < p.W; w += STEP_THREADS) smask[w] = 0u;
-        __syncthreads();
-        for (int i = cb + threadIdx.x; i < ce; i += STEP_THREADS) {
-            int32_t t = __ldg(p.node_tok + i);
-            atomicOr(&smask[t >> 5], 1u << (t & 31));
-        }
-    }
-    __syncthreads();
-}
-
 // position of token t among the sorted children [cb, ce) of a node, found by one warp: each round
 // 32 lanes probe evenly spaced keys and keep the sub-range that can still hold t.  -1 if absent.
 __device__ int32_t warp_find_child(const int32_t* __restrict__ node_tok, int32_t cb, int32_t ce, int32_t t) {
@@ -356,99 +397,120 @@ __device__ int32_t warp_find_child(const int32_t* __restrict__ node_tok, int32_t
 }
 
 // ---- streaming loops ---------------------------------------------------------------------------
-// Bulk-copy ring: returns false if an mbarrier wait gave up.
+struct RingGeom {
+    const char* rowp;        // the row's logits
+    const char* gmask;       // the row's prebuilt mask (dense rows), else nullptr
+    uint32_t vec_bytes;      // bytes of whole 16-byte vectors in the row
+    uint32_t mask_bytes;     // bytes of the mask row that may be read (a multiple of 16)
+    uint32_t slice;          // mask bytes per full chunk
+    uint32_t ring_s, full_s; // shared-memory addresses of the ring and of the full barriers
+};
+
+// copy chunk c of the row (and, for dense rows, the mask slice covering it) into ring stage s and
+// arm the stage's full barrier (one thread)
+__device__ __forceinline__ void ring_issue(const RingGeom& g, int c, int s, bool with_mask) {
+    const uint32_t off = uint32_t(c) * CHUNK_BYTES;
+    const uint32_t bytes = min(uint32_t(CHUNK_BYTES), g.vec_bytes - off);
+    const uint32_t bar = g.full_s + 8u * s;
+    const uint32_t dst = g.ring_s + uint32_t(s) * STAGE_BYTES;
+    uint32_t mbytes = 0, moff = 0;
+    if (with_mask) {
+        moff = uint32_t(c) * g.slice;
+        mbytes = moff < g.mask_bytes ? min(g.slice, g.mask_bytes - moff) : 0u;
+    }
+    mbar_expect_tx(bar, bytes + mbytes);
+    bulk_g2s(dst, g.rowp + off, bytes, bar);
+    if (mbytes) bulk_g2s(dst + CHUNK_BYTES, g.gmask + moff, mbytes, bar);
+}
+
+// Bulk-copy ring.  Chunk c of the row lives in stage c % STAGES.  The logits of the first STAGES
+// chunks are issued by the kernel's prologue before the prefix index is read, and (for dense rows)
+// their mask slices right after it, on a barrier of their own (mask0).  Then thread 0 keeps
+// STAGES-1 chunks in flight: after every warp has copied chunk c-1 out of its stage (empty
+// barrier), that stage is refilled with chunk c-1+STAGES.  Returns false if a wait gave up.
 template <int DT, bool DENSE>
-__device__ bool stream_ring(Acc& a, const RowCtx& r, const char* rowp, int V, unsigned char* ring,
-                            uint64_t* full_bar, uint64_t* empty_bar, const uint32_t* smask) {
+__device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const RingGeom& g, int V,
+                            const unsigned char* ring, uint32_t empty_s, uint32_t mask0_s) {
     using E = Elem<DT>;
     constexpr int EPV = E::EPV;
     const int tid = threadIdx.x, lane = tid & 31;
     const int nvec = V / EPV;
-    const uint32_t vec_bytes = uint32_t(nvec) * 16u;
-    const int n_chunks = int((vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
-    const uint32_t ring_s = smem_u32(ring);
+    const int n_chunks = int((g.vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
+    const int n_full = int(g.vec_bytes / CHUNK_BYTES);
     bool ok = true;
 
-    auto issue = [&](int c) {
-        const int s = c % STAGES;
-        const uint32_t off = uint32_t(c) * CHUNK_BYTES;
-        const uint32_t bytes = min(uint32_t(CHUNK_BYTES), vec_bytes - off);
-        const uint32_t bar = smem_u32(&full_bar[s]);
-        mbar_expect_tx(bar, bytes);
-        bulk_g2s(ring_s + uint32_t(s) * CHUNK_BYTES, rowp + off, bytes, bar);
-    };
-    if (tid == 0) {
-        for (int c = 0; c < STAGES && c < n_chunks; ++c) issue(c);
+    // the mask slices of the first STAGES chunks were copied separately (see the kernel's prologue)
+    if constexpr (DENSE) {
+        if (!__all_sync(0xffffffffu, mbar_wait(mask0_s, 0u))) return false;
     }
+
+    int s = 0, sp = STAGES - 1;          // stage of chunk c and of chunk c-1
+    uint32_t ph = 0, php = 1;            // their phase parities (php is only used from c = 1 on)
     for (int c = 0; c < n_chunks; ++c) {
-        const int s = c % STAGES;
-        const uint32_t use = uint32_t(c / STAGES);     // how often stage s was used before
         // the give-up decision is taken per warp, so that all lanes leave the loop together
-        if (!__all_sync(0xffffffffu, mbar_wait(smem_u32(&full_bar[s]), use & 1u))) { ok = false; break; }
+        if (!__all_sync(0xffffffffu, mbar_wait(g.full_s + 8u * s, ph))) { ok = false; break; }
+        const unsigned char* stage_b = ring + s * STAGE_BYTES;
+        const uint4* stage = reinterpret_cast<const uint4*>(stage_b);
         uint4 raw[VPT];
+        uint32_t bits[VPT];
+        const bool full = c < n_full;
+        const int g0 = c * CHUNK_VECS + tid;
 #pragma unroll
         for (int j = 0; j < VPT; ++j) {
-            const int in_chunk = j * STEP_THREADS + tid;
-            const int g = c * (CHUNK_BYTES / 16) + in_chunk;
-            if (g < nvec) raw[j] = *reinterpret_cast<const uint4*>(ring + s * CHUNK_BYTES + in_chunk * 16);
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(smem_u32(&empty_bar[s]));
-        // refill the stage released one iteration ago (every warp has long passed it)
-        if (tid == 0 && c >= 1 && c - 1 + STAGES < n_chunks) {
-            const int sp = (c - 1) % STAGES;
-            const uint32_t usep = uint32_t((c - 1) / STAGES);
-            if (!mbar_wait(smem_u32(&empty_bar[sp]), usep & 1u)) ok = false;
-            else issue(c - 1 + STAGES);
-        }
-        if (c == 0 && tid < nvec) {
-            float x[EPV];
-            E::unpack(raw[0], x);
-            float mx = x[0];
-#pragma unroll
-            for (int j = 1; j < EPV; ++j) mx = fmaxf(mx, x[j]);
-            set_reference(a, r, mx);
-            if constexpr (DENSE) update_bound(a, r);
-        }
-#pragma unroll
-        for (int j = 0; j < VPT; ++j) {
-            const int g = c * (CHUNK_BYTES / 16) + j * STEP_THREADS + tid;
-            if (g < nvec) {
-                float x[EPV];
-                E::unpack(raw[j], x);
-                consume<EPV, DENSE>(a, r, x, g * EPV, smask);
+            bits[j] = 0;
+            if (full || g0 + j * STEP_THREADS < nvec) {
+                raw[j] = stage[j * STEP_THREADS + tid];
+                if constexpr (DENSE) {
+                    const int iv = j * STEP_THREADS + tid;       // vector index inside the chunk
+                    if constexpr (EPV == 8) bits[j] = stage_b[CHUNK_BYTES + iv];
+                    else bits[j] = (uint32_t(stage_b[CHUNK_BYTES + (iv >> 1)]) >> ((iv & 1) * 4)) & 0xFu;
+                }
             }
         }
+        __syncwarp();
+        if (lane == 0) mbar_arrive(empty_s + 8u * s);
+        if (tid == 0 && c >= 1 && c - 1 + STAGES < n_chunks) {
+            if (!mbar_wait(empty_s + 8u * sp, php)) ok = false;
+            else ring_issue(g, c - 1 + STAGES, sp, DENSE);
+        }
+        if (c == 0 && tid < nvec) {
+            float2 x[EPV / 2];
+            E::unpack(raw[0], x);
+            float mx = fmaxf(x[0].x, x[0].y);
+#pragma unroll
+            for (int i = 1; i < EPV / 2; ++i) mx = fmaxf(mx, fmaxf(x[i].x, x[i].y));
+            set_reference(a, r, mx);
+        }
+#pragma unroll
+        for (int j = 0; j < VPT; ++j)
+            if (full || g0 + j * STEP_THREADS < nvec)
+                consume_vec<DT, DENSE>(a, r, rk, raw[j], (g0 + j * STEP_THREADS) * EPV, bits[j]);
+        if constexpr (DENSE) share_bound(a);
+        sp = s; php = ph;
+        if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
     // ragged tail: V not a multiple of the vector width
     const int v = nvec * EPV + tid;
-    if (v < V) {
-        float x[1] = {E::load(rowp, v)};
-        if (!a.touched) { set_reference(a, r, x[0]); if constexpr (DENSE) update_bound(a, r); }
-        consume<1, DENSE>(a, r, x, v, smask);
-    }
+    if (v < V) consume_one<DENSE>(a, r, rk, E::load(g.rowp, v), v, reinterpret_cast<const uint32_t*>(g.gmask));
     return ok;
 }
 
 template <int DT, bool DENSE>
-__device__ void stream_scalar(Acc& a, const RowCtx& r, const char* rowp, int V, const uint32_t* smask) {
+__device__ void stream_scalar(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp, int V,
+                              const uint32_t* gmask) {
     using E = Elem<DT>;
-    for (int v = threadIdx.x; v < V; v += STEP_THREADS) {
-        float x[1] = {E::load(rowp, v)};
-        if (!a.touched) { set_reference(a, r, x[0]); if constexpr (DENSE) update_bound(a, r); }
-        consume<1, DENSE>(a, r, x, v, smask);
-    }
+    for (int v = threadIdx.x; v < V; v += STEP_THREADS) consume_one<DENSE>(a, r, rk, E::load(rowp, v), v, gmask);
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
 template <int DT, bool RING>
-__global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepParams p) {
+__global__ void __launch_bounds__(STEP_THREADS, DISC_MIN_BLOCKS)
+disc_step_kernel(const __grid_constant__ StepParams p) {
     using E = Elem<DT>;
-    extern __shared__ __align__(128) unsigned char dyn_smem[];
-    unsigned char* ring = dyn_smem;                                             // RING_BYTES (RING only)
-    uint32_t* smask = reinterpret_cast<uint32_t*>(dyn_smem + (RING ? RING_BYTES : 0));
+    extern __shared__ __align__(128) unsigned char ring[];        // RING_BYTES (RING only)
     __shared__ __align__(8) uint64_t full_bar[STAGES];
     __shared__ __align__(8) uint64_t empty_bar[STAGES];
+    __shared__ __align__(8) uint64_t mask0_bar;
     __shared__ float red_f[6][STEP_WARPS];
     __shared__ int32_t red_i[2][STEP_WARPS];
     __shared__ float scratch[STEP_WARPS];
@@ -463,6 +525,28 @@ __global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepPa
         if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_DONE; }
         return;
     }
+    // Start streaming before anything else: the first ring stage fills while the index is read.
+    RingGeom g;
+    g.rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
+    g.gmask = nullptr;
+    g.vec_bytes = uint32_t(p.V / E::EPV) * 16u;
+    g.mask_bytes = uint32_t(p.Wp) * 4u;
+    g.slice = uint32_t(CHUNK_VECS * E::EPV / 8);
+    g.ring_s = smem_u32(ring);
+    g.full_s = smem_u32(full_bar);
+    const int n_chunks = int((g.vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
+    if (RING && tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            mbar_init(smem_u32(&full_bar[s]), 1);
+            mbar_init(smem_u32(&empty_bar[s]), STEP_WARPS);
+        }
+        mbar_init(smem_u32(&mask0_bar), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        for (int k = 0; k < STAGES && k < n_chunks; ++k) ring_issue(g, k, k, false);
+    }
+    if (tid == 0) s_fault = 0;
+
     const int32_t node = p.node[row];
     int32_t cb = 0, ce = 0;
     if (node >= 0 && int64_t(node) < p.M) { cb = __ldg(p.child_begin + node); ce = __ldg(p.child_begin + node + 1); }
@@ -473,52 +557,77 @@ __global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepPa
             bool leaf = node > 0 && int64_t(node) < p.M;
             p.status_out[row] = leaf ? DISC_ROW_DONE : DISC_ROW_DEAD;
             if (leaf) p.done[row] = 1;
+            // the copies already in flight must land before the block's shared memory is released
+            if (RING)
+                for (int k = 0; k < STAGES && k < n_chunks; ++k) mbar_wait(smem_u32(&full_bar[k]), 0u);
         }
         return;
     }
 
-    if (RING) {
-        if (tid == 0) {
-            for (int s = 0; s < STAGES; ++s) {
-                mbar_init(smem_u32(&full_bar[s]), 1);
-                mbar_init(smem_u32(&empty_bar[s]), STEP_WARPS);
+    // dense rows: locate the prebuilt mask row (root, or a heavy node) and fetch the mask slices of
+    // the chunks already in flight
+    if (tid == 0) {
+        int32_t h = -2;                                   // -2: not dense
+        if (node == 0) h = -1;                            // -1: the root's row
+        else if (c > DISC_HEAVY_MIN) { h = heavy_index(p.heavy_nodes, p.n_heavy, node); if (h < 0) h = -2; }
+        s_tmp = h;
+        if (RING && h != -2) {
+            const char* gm = reinterpret_cast<const char*>(h == -1 ? p.root_mask : p.heavy_masks + size_t(h) * p.Wp);
+            uint32_t total = 0;
+            for (int k = 0; k < STAGES && k < n_chunks; ++k) {
+                const uint32_t moff = uint32_t(k) * g.slice;
+                total += moff < g.mask_bytes ? min(g.slice, g.mask_bytes - moff) : 0u;
             }
-            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            const uint32_t bar = smem_u32(&mask0_bar);
+            mbar_expect_tx(bar, total);
+            for (int k = 0; k < STAGES && k < n_chunks; ++k) {
+                const uint32_t moff = uint32_t(k) * g.slice;
+                const uint32_t mb = moff < g.mask_bytes ? min(g.slice, g.mask_bytes - moff) : 0u;
+                if (mb) bulk_g2s(g.ring_s + uint32_t(k) * STAGE_BYTES + CHUNK_BYTES, gm + moff, mb, bar);
+            }
         }
     }
-    if (tid == 0) s_fault = 0;
     __syncthreads();
+    const int32_t hsel = s_tmp;
+    const bool dense = hsel != -2;
+    const uint32_t* gmask = !dense ? nullptr : (hsel == -1 ? p.root_mask : p.heavy_masks + size_t(hsel) * p.Wp);
+    g.gmask = reinterpret_cast<const char*>(gmask);
 
-    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
     RowCtx r;
-    r.c2 = p.c2; r.inv_t = p.inv_t; r.key = p.key; r.step = p.step; r.row = uint32_t(p.row_base + uint32_t(row));
-    r.xref = E::load(rowp, 0);
+    r.c2 = p.c2; r.inv_t = p.inv_t; r.step = p.step; r.row = uint32_t(p.row_base + uint32_t(row));
+    r.xref = E::load(g.rowp, 0);
     if (!(fabsf(r.xref) < CUDART_INF_F)) r.xref = 0.f;
-    const bool dense = (c > DISC_HEAVY_MIN) || (p.mask_out != nullptr);
 
     Acc a;
     MS ok{-CUDART_INF_F, 0.f};
     bool poisoned = false;
 
-    if (dense) {
-        build_mask(smask, p, node, cb, ce, &s_tmp);
-        if (p.mask_out) {
-            uint32_t* mo = p.mask_out + size_t(row) * p.W;
-            for (int w = tid; w < p.W; w += STEP_THREADS) mo[w] = smask[w];
+    if (p.mask_out) {
+        // optional output of the valid-set mask
+        uint32_t* mo = p.mask_out + size_t(row) * p.W;
+        if (dense) {
+            for (int w = tid; w < p.W; w += STEP_THREADS) mo[w] = __ldg(gmask + w);
+        } else {
+            for (int w = tid; w < p.W; w += STEP_THREADS) mo[w] = 0u;
+            __syncthreads();
+            for (int i = cb + tid; i < ce; i += STEP_THREADS) {
+                const int32_t t = __ldg(p.node_tok + i);
+                atomicOr(&mo[t >> 5], 1u << (t & 31));
+            }
         }
-    } else {
+    }
+    if (!dense) {
         // gather path: the few allowed logits are read directly
         for (int i = tid; i < c; i += STEP_THREADS) {
             const int32_t v = __ldg(p.node_tok + cb + i);
-            const float x = E::load(rowp, v);
+            const float x = E::load(g.rowp, v);
             // sum of 2^(x*c2) kept as 2^m * s; fma(x, c2, -m) is the exact product minus the
             // reference, so a large common offset of the logits costs no accuracy
             const float y = x * p.c2;
             if (!(y < CUDART_INF_F)) poisoned = true;                 // NaN or +inf: careful path
             else if (y > ok.m) { ok.s = ok.s * exp2f(ok.m - y) + exp2f(fmaf(x, p.c2, -y)); ok.m = y; }
             else if (y != -CUDART_INF_F) ok.s += exp2f(fmaf(x, p.c2, -ok.m));
-            const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, r.key);
+            const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, p.rk);
             const float score = gumbel_score(x, r.xref, r.inv_t, pick_word(w4, v & 3));
             if (score > a.best.score) { a.best.score = score; a.best.tok = v; a.best.child = cb + i; }
         }
@@ -527,20 +636,20 @@ __global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepPa
     // ---- stream the row
     bool waits_ok = true;
     if (RING) {
-        waits_ok = dense ? stream_ring<DT, true>(a, r, rowp, p.V, ring, full_bar, empty_bar, smask)
-                         : stream_ring<DT, false>(a, r, rowp, p.V, ring, full_bar, empty_bar, smask);
+        waits_ok = dense ? stream_ring<DT, true>(a, r, p.rk, g, p.V, ring, smem_u32(empty_bar), smem_u32(&mask0_bar))
+                         : stream_ring<DT, false>(a, r, p.rk, g, p.V, ring, smem_u32(empty_bar), smem_u32(&mask0_bar));
     } else {
-        if (dense) stream_scalar<DT, true>(a, r, rowp, p.V, smask);
-        else stream_scalar<DT, false>(a, r, rowp, p.V, smask);
+        if (dense) stream_scalar<DT, true>(a, r, p.rk, g.rowp, p.V, gmask);
+        else stream_scalar<DT, false>(a, r, p.rk, g.rowp, p.V, gmask);
     }
     if (!waits_ok) s_fault = 1;
 
-    MS all = a.touched ? MS{a.mref, a.s_all0 + a.s_all1} : MS{-CUDART_INF_F, 0.f};
-    if (dense) ok = a.touched ? MS{a.mref, a.s_ok} : MS{-CUDART_INF_F, 0.f};
+    MS all = a.touched ? MS{a.mref, (a.sa.x + a.sa.y) + (a.sb.x + a.sb.y)} : MS{-CUDART_INF_F, 0.f};
+    if (dense) ok = a.touched ? MS{a.mref, a.ok2.x + a.ok2.y} : MS{-CUDART_INF_F, 0.f};
     if (poisoned) ok.s = CUDART_NAN_F;
     Best best = a.best;
 
-    const int any_lost = __syncthreads_or(a.lost ? 1 : 0);
+    __syncthreads();
     if (s_fault) {
         // A bulk copy never signalled completion.  Report it and leave the row untouched; give
         // outstanding copies a bounded time to land before the block's shared memory is released.
@@ -591,30 +700,41 @@ __global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepPa
         fin[0] = all.m; fin[1] = all.s; fin[2] = ok.m; fin[3] = ok.s;
         const float l2_all = all.m + log2f(all.s);
         const float l2_ok = ok.m + log2f(ok.s);
-        // the fast sums are trusted only when both are finite and no allowed term was lost
-        s_flag = (fabsf(l2_all) < CUDART_INF_F && fabsf(l2_ok) < CUDART_INF_F && !any_lost) ? 0 : 1;
+        // The fast sums are trusted when both are finite.  In the dense path the valid-set sum
+        // shares each thread's reference with the full sum, so an allowed term 2^-126 below a
+        // thread's reference is flushed to zero (and its token skipped by the bound).  all.m is the
+        // largest reference; while log2(valid mass) >= all.m - 60 every flushed term is below
+        // 2^-49 of the valid sum even if all 2^17 of them were flushed, and no flushed token can
+        // win (its score trails the best allowed token by more than the largest noise).
+        bool trust = fabsf(l2_all) < CUDART_INF_F && fabsf(l2_ok) < CUDART_INF_F;
+        if (dense && !(l2_ok >= all.m - MASS_FLOOR_LOG2)) trust = false;
+        s_flag = trust ? 0 : 1;
         red_f[4][0] = best.score; red_i[0][0] = best.tok; red_i[1][0] = best.child;
     }
     __syncthreads();
 
     if (s_flag) {
-        // ---- careful path: plain two-pass log-sum-exp over the row with an explicit mask and
-        // separate maxima for the full row and for the valid set; in the dense path the scores of
-        // all allowed tokens are evaluated exactly again (its skip bound relies on terms that did
-        // not underflow)
-        if (!dense) build_mask(smask, p, node, cb, ce, &s_tmp);
+        // ---- careful path: plain two-pass log-sum-exp with separate maxima for the full row and
+        // for the valid set.  Dense rows test the prebuilt mask and evaluate the score of every
+        // allowed token exactly again; gather rows walk their child list (their scores were exact).
         float mx_all = -CUDART_INF_F, mx_ok = -CUDART_INF_F;
         int nan_all = 0, nan_ok = 0;
         Best cbest{-CUDART_INF_F, -1, -1};
         for (int v = tid; v < p.V; v += STEP_THREADS) {
-            const float x = E::load(rowp, v);
-            const bool allowed = (smask[v >> 5] >> (v & 31)) & 1u;
+            const float x = E::load(g.rowp, v);
+            const bool allowed = dense && mask_bit(gmask, v);
             if (x != x) { nan_all = 1; nan_ok |= allowed; }
             else { mx_all = fmaxf(mx_all, x); if (allowed) mx_ok = fmaxf(mx_ok, x); }
-            if (allowed && dense) {
-                const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, r.key);
+            if (allowed) {
+                const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, p.rk);
                 const float score = gumbel_score(x, r.xref, r.inv_t, pick_word(w4, v & 3));
                 if (score > cbest.score) { cbest.score = score; cbest.tok = v; }
+            }
+        }
+        if (!dense) {
+            for (int i = tid; i < c; i += STEP_THREADS) {
+                const float x = E::load(g.rowp, __ldg(p.node_tok + cb + i));
+                if (x != x) nan_ok = 1; else mx_ok = fmaxf(mx_ok, x);
             }
         }
         mx_all = block_max(mx_all, scratch);
@@ -625,10 +745,13 @@ __global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepPa
         const float r_all = mx_all * p.c2, r_ok = mx_ok * p.c2;
         float sum_all = 0.f, sum_ok = 0.f;
         for (int v = tid; v < p.V; v += STEP_THREADS) {
-            const float x = E::load(rowp, v);
-            const bool allowed = (smask[v >> 5] >> (v & 31)) & 1u;
+            const float x = E::load(g.rowp, v);
             if (fin_all) sum_all += exp2f(fmaf(x, p.c2, -r_all));
-            if (fin_ok && allowed) sum_ok += exp2f(fmaf(x, p.c2, -r_ok));
+            if (fin_ok && dense && mask_bit(gmask, v)) sum_ok += exp2f(fmaf(x, p.c2, -r_ok));
+        }
+        if (!dense && fin_ok) {
+            for (int i = tid; i < c; i += STEP_THREADS)
+                sum_ok += exp2f(fmaf(E::load(g.rowp, __ldg(p.node_tok + cb + i)), p.c2, -r_ok));
         }
         sum_all = block_sum(sum_all, scratch);
         sum_ok = block_sum(sum_ok, scratch);
@@ -678,7 +801,7 @@ __global__ void __launch_bounds__(STEP_THREADS, 3) disc_step_kernel(const StepPa
             uint8_t st = 0;
             if (!f_all) st |= DISC_ROW_NONFINITE;
             if (!f_ok) st |= DISC_ROW_NOMASS;
-            const float xt = E::load(rowp, tok);
+            const float xt = E::load(g.rowp, tok);
             const float logq = f_ok ? (fmaf(xt, p.c2, -K.m) - lg_ok) * LN2_F : (xt * p.c2 - l2_ok) * LN2_F;
             const float logp = f_all ? (fmaf(xt, p.c2, -A.m) - lg_all) * LN2_F : (xt * p.c2 - l2_all) * LN2_F;
             const int32_t d = p.depth[row];
@@ -705,11 +828,12 @@ __global__ void k_state_init(int64_t n, int32_t N, int32_t* node, int32_t* lo, i
     node[i] = 0; lo[i] = 0; hi[i] = N; depth[i] = 0; logw[i] = 0.f; done[i] = 0;
 }
 
-__global__ void k_sampling_uniforms(PhiloxKey key, uint32_t step, uint32_t row, int32_t v0, int32_t n, float* out) {
+__global__ void k_sampling_uniforms(PhiloxRoundKeys rk, uint32_t step, uint32_t row, int32_t v0, int32_t n,
+                                    float* out) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
     uint32_t v = uint32_t(v0 + i);
-    uint4 r = philox4x32_10(v >> 2, step, row, 0u, key);
+    uint4 r = philox4x32_10(v >> 2, step, row, 0u, rk);
     out[i] = uniform_from_bits(pick_word(r, v & 3));
 }
 
@@ -748,24 +872,22 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     if (ld < s->V || row_base < 0 || (seq_tokens && seq_ld <= 0)) return DISC_ERR_ARG;
     if (!(inv_temperature > 0.f) || !(inv_temperature <= 3.0e38f)) return DISC_ERR_ARG;
     if (dtype != DISC_F32 && dtype != DISC_BF16) return DISC_ERR_UNSUPPORTED;
-    const size_t mask_bytes = (size_t(s->W) * 4 + 15) & ~size_t(15);
-    if (mask_bytes > 160 * 1024) return DISC_ERR_UNSUPPORTED;
 
     StepParams p;
     p.logits = logits; p.ld = ld; p.inv_t = inv_temperature; p.c2 = inv_temperature * LOG2E_F;
-    p.key = philox_key(seed); p.step = step; p.row_base = uint32_t(row_base);
+    p.rk = philox_round_keys(seed); p.step = step; p.row_base = uint32_t(row_base);
     p.node = node; p.lo = lo; p.hi = hi; p.depth = depth; p.logw = logw; p.done = done;
     p.token_out = token_out; p.seq_tokens = seq_tokens; p.seq_ld = seq_ld;
     p.logq_out = logq_out; p.logp_out = logp_out; p.mask_out = mask_out; p.status_out = status_out;
     p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
     p.root_child = s->root_child; p.root_mask = s->root_mask;
     p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
-    p.V = s->V; p.W = s->W; p.M = s->M;
+    p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.M = s->M;
 
     const size_t esize = dtype == DISC_F32 ? 4 : 2;
     // the bulk-copy ring needs 16-byte aligned rows; other layouts take the scalar path
     const bool ring = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
-    const size_t smem = mask_bytes + (ring ? RING_BYTES : 0);
+    const size_t smem = ring ? RING_BYTES : 0;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (dtype == DISC_F32) return ring ? launch_step<DISC_F32, true>(p, n, smem, st) : launch_step<DISC_F32, false>(p, n, smem, st);
     return ring ? launch_step<DISC_BF16, true>(p, n, smem, st) : launch_step<DISC_BF16, false>(p, n, smem, st);
@@ -775,8 +897,8 @@ int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t v
                            void* stream) {
     if (n < 0 || v0 < 0 || (n > 0 && !out)) return DISC_ERR_ARG;
     if (n == 0) return DISC_OK;
-    k_sampling_uniforms<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(philox_key(seed), step, row,
-                                                                                       v0, n, out);
+    k_sampling_uniforms<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(philox_round_keys(seed),
+                                                                                       step, row, v0, n, out);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }
