@@ -62,7 +62,7 @@ def lib():
         L.oracle_mask.restype = None
         L.oracle_step.argtypes = [vp, vp, C.c_int, i64, i64, C.c_float, u64, u32, vp,
                                   vp, i32, vp, vp, vp,
-                                  vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
+                                  vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
         L.oracle_step.restype = None
         L.oracle_resample.argtypes = [vp, i32, i32, u64, vp, vp, vp, vp, vp, vp]
         L.oracle_resample.restype = None
@@ -73,8 +73,10 @@ def lib():
         L.oracle_decode_markov.restype = C.c_int
         L.oracle_philox4x32_10.argtypes = [vp, vp, vp]
         L.oracle_philox4x32_10.restype = None
-        L.oracle_gumbel_uniform.argtypes = [u64, u32, u32, u32]
-        L.oracle_gumbel_uniform.restype = C.c_double
+        L.oracle_group_uniform.argtypes = [u64, u32, u32, u32]
+        L.oracle_group_uniform.restype = C.c_double
+        L.oracle_ingroup_uniform.argtypes = [u64, u32, u32, u32]
+        L.oracle_ingroup_uniform.restype = C.c_double
         L.oracle_resample_uniform.argtypes = [u64, u32]
         L.oracle_resample_uniform.restype = C.c_double
         L.oracle_accept_uniform.argtypes = [u64, u32, u32]
@@ -169,7 +171,8 @@ class OracleSet:
             "token": np.empty(n, np.int32), "lo": np.empty(n, np.int32), "hi": np.empty(n, np.int32),
             "done": np.empty(n, np.uint8), "log_mass": np.empty(n), "lse_all": np.empty(n),
             "lse_ok": np.empty(n), "logq": np.empty(n), "logp": np.empty(n), "best": np.empty(n),
-            "second": np.empty(n), "alt": np.empty(n), "n_children": np.empty(n, np.int32),
+            "second": np.empty(n), "alt": np.empty(n), "ingroup_gap": np.empty(n),
+            "n_children": np.empty(n, np.int32),
             "status": np.empty(n, np.uint8),
         }
         lib().oracle_step(self._h, _p(logits), int(dtype), logits.shape[1], n, float(inv_temperature),
@@ -177,7 +180,7 @@ class OracleSet:
                           _p(done), _p(alt_token),
                           _p(o["token"]), _p(o["lo"]), _p(o["hi"]), _p(o["done"]), _p(o["log_mass"]),
                           _p(o["lse_all"]), _p(o["lse_ok"]), _p(o["logq"]), _p(o["logp"]),
-                          _p(o["best"]), _p(o["second"]), _p(o["alt"]), _p(o["n_children"]),
+                          _p(o["best"]), _p(o["second"]), _p(o["alt"]), _p(o["ingroup_gap"]), _p(o["n_children"]),
                           _p(o["status"]), int(n_threads))
         return o
 
@@ -228,8 +231,14 @@ def philox4x32_10(ctr, key):
     return out
 
 
-def gumbel_uniform(seed, step, row, v):
-    return lib().oracle_gumbel_uniform(int(seed), int(step), int(row), int(v))
+def group_uniform(seed, step, row, group):
+    """Uniform behind the Gumbel noise of token group `group` (= token id >> 3)."""
+    return lib().oracle_group_uniform(int(seed), int(step), int(row), int(group))
+
+
+def ingroup_uniform(seed, step, row, group):
+    """Uniform of the inverse-CDF draw inside the winning group."""
+    return lib().oracle_ingroup_uniform(int(seed), int(step), int(row), int(group))
 
 
 def resample_uniform(seed, query):

@@ -26,8 +26,10 @@
 // Readings where the paper is silent (same list as the design notes):
 //   * S must be prefix-free (fixed length, or every member closed by an EOS
 //     that is an ordinary token); then "a in S" is "the node is a leaf".
-//   * sampling is Gumbel-max over the allowed tokens with one uniform per
-//     (row, step, token id) from Philox4x32-10; ties go to the lowest id.
+//   * sampling is exact and two-stage: Gumbel-max over groups of 8 consecutive
+//     token ids (group score = log of the group's allowed mass + Gumbel noise,
+//     one Philox4x32-10 uniform per (row, step, group), ties to the lowest
+//     group), then an inverse-CDF draw inside the winning group.
 //   * all floating point here is fp64.
 //
 // Parity pins for these functions live in tests/test_oracle_*.py.  The Philox
@@ -219,13 +221,24 @@ void philox4x32_10(const uint32_t c_in[4], const uint32_t k_in[2], uint32_t out[
 // exactly representable in fp32 (odd numerators below 2^24)
 double uniform23(uint32_t r) { return (double(r >> 9) + 0.5) * (1.0 / 8388608.0); }
 
-// domain 0: one uniform per (row, step, token id)
-double gumbel_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t v) {
-    uint32_t ctr[4] = {v >> 2, step, row, 0u};
+// Sampling works on groups of 8 consecutive token ids (group G = v >> 3); see step_row.
+// domain 0: one uniform per (row, step, group).  Groups are spread over Philox counters so that the
+// four words of one counter belong to groups 256 apart: counter word 0 = ((G>>10)<<8) | (G & 255),
+// output word (G >> 8) & 3.  (Any bijection would do; this one is fixed by this build's convention.)
+double group_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t G) {
+    uint32_t ctr[4] = {((G >> 10) << 8) | (G & 255u), step, row, 0u};
     uint32_t key[2] = {uint32_t(seed), uint32_t(seed >> 32)};
     uint32_t out[4];
     philox4x32_10(ctr, key, out);
-    return uniform23(out[v & 3]);
+    return uniform23(out[(G >> 8) & 3u]);
+}
+// domain 3: one uniform per (row, step, group) for the draw inside the winning group
+double ingroup_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t G) {
+    uint32_t ctr[4] = {G, step, row, 3u};
+    uint32_t key[2] = {uint32_t(seed), uint32_t(seed >> 32)};
+    uint32_t out[4];
+    philox4x32_10(ctr, key, out);
+    return uniform23(out[0]);
 }
 // domain 1: one uniform per query for the K-way draw
 double resample_uniform(uint64_t seed, uint32_t query) {
@@ -259,7 +272,8 @@ struct StepOut {
     int32_t token = -1, lo = -1, hi = -1;
     uint8_t done = 0, status = 0;
     double log_mass = QNAN, lse_all = QNAN, lse_ok = QNAN, logq = QNAN, logp = QNAN;
-    double best = QNAN, second = QNAN, alt = QNAN;
+    double best = QNAN, second = QNAN, alt = QNAN;      // group scores: winner, runner-up, alt token's group
+    double ingroup_gap = std::numeric_limits<double>::infinity();   // see step_row, stage (2)
     int32_t n_children = 0;
 };
 
@@ -291,19 +305,54 @@ StepOut step_row(const Trie& T, int32_t node, const void* logits, int dtype, int
     for (int32_t v = 0; v < T.V; ++v) all.add(load_logit(logits, dtype, base + v) * inv_t);
     o.lse_all = all.value();
 
+    // Sampling from P.mask / |P.mask|_1 (Algorithm 1, line 7), exact, in two stages:
+    //  (1) Gumbel-max over groups of 8 consecutive token ids (G = v >> 3): the score of a group is
+    //      log(sum of e^{z_v} over its allowed tokens) - log(-log u_G); the largest score wins, the
+    //      lowest group on an exact tie; NaN and -inf scores never win.  (The maximum of
+    //      Gumbel-perturbed scores of a set of tokens is distributed as the perturbed log of their
+    //      total mass, so the winning group is drawn with probability mass_G / total mass.)
+    //  (2) inside the winning group, the smallest allowed token whose inclusive cumulative weight
+    //      exceeds u' * mass_G (inverse CDF, tokens in ascending id).
     Lse ok;
+    struct Member { int32_t child, tok; double z; };
+    std::vector<Member> cur, win;
+    int32_t cur_g = -1;
     double best = NEG_INF, second = NEG_INF;
-    int32_t best_child = T.first_child[node];                  // lowest id unless beaten
+    auto close_group = [&]() {
+        if (cur.empty()) return;
+        Lse mass;
+        for (const Member& m : cur) mass.add(m.z);
+        double u = group_uniform(seed, step, row, uint32_t(cur_g));
+        double score = mass.value() + (-std::log(-std::log(u)));
+        for (const Member& m : cur) if (m.tok == alt_token) o.alt = score;
+        if (score > best) { second = best; best = score; win = cur; }
+        else if (score > second) second = score;
+        cur.clear();
+    };
     for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c]) {
         ++o.n_children;
         int32_t v = T.tok[c];
         double z = load_logit(logits, dtype, base + v) * inv_t;
         ok.add(z);
-        double u = gumbel_uniform(seed, step, row, uint32_t(v));
-        double score = z + (-std::log(-std::log(u)));
-        if (v == alt_token) o.alt = score;
-        if (score > best) { second = best; best = score; best_child = c; }
-        else if (score > second) second = score;
+        if ((v >> 3) != cur_g) { close_group(); cur_g = v >> 3; }
+        cur.push_back({c, v, z});
+    }
+    close_group();
+    int32_t best_child = T.first_child[node];                  // lowest id unless a group wins
+    if (!win.empty()) {
+        double zmax = NEG_INF, total = 0.0;
+        for (const Member& m : win) if (m.z > zmax) zmax = m.z;
+        std::vector<double> C(win.size());
+        for (size_t i = 0; i < win.size(); ++i) { total += std::exp(win[i].z - zmax); C[i] = total; }
+        size_t pick = 0;
+        if (std::isfinite(total) && total > 0.0) {
+            double target = ingroup_uniform(seed, step, row, uint32_t(win[0].tok >> 3)) * total;
+            pick = win.size() - 1;
+            for (size_t i = 0; i < win.size(); ++i) if (C[i] > target) { pick = i; break; }
+            double below = pick > 0 ? C[pick - 1] : 0.0;
+            o.ingroup_gap = std::min(std::fabs(target - below), std::fabs(C[pick] - target)) / total;
+        }
+        best_child = win[pick].child;
     }
     o.lse_ok = ok.value();
     o.log_mass = o.lse_ok - o.lse_all;
@@ -417,14 +466,17 @@ void oracle_mask(const void* h, const int32_t* prefix, int32_t prefix_ld, const 
 // One decoding step for n rows.  Row i's prefix is prefix[i*prefix_ld .. +depth[i]); its logits are
 // logits[i*ld .. +V); its RNG row index is row_ids[i] (i when row_ids is null).  Rows with done[i]
 // != 0 are skipped (token -1, status 8).  Every output array has n entries; alt_token is optional:
-// alt_score[i] is this oracle's perturbed score of alt_token[i] (NaN if it is not allowed).
+// alt_score[i] is this oracle's perturbed score of the group of alt_token[i] (NaN if that token is
+// not allowed); best/second are the winning and runner-up group scores; ingroup_gap[i] is the
+// distance of the in-group threshold to the nearest boundary of the chosen token's interval, as a
+// fraction of the group's mass (for near-tie accounting).
 void oracle_step(const void* h, const void* logits, int dtype, int64_t ld, int64_t n,
                  float inv_temperature, uint64_t seed, uint32_t step, const int64_t* row_ids,
                  const int32_t* prefix, int32_t prefix_ld, const int32_t* depth, const uint8_t* done,
                  const int32_t* alt_token,
                  int32_t* token, int32_t* lo, int32_t* hi, uint8_t* done_out,
                  double* log_mass, double* lse_all, double* lse_ok, double* logq, double* logp,
-                 double* best_score, double* second_score, double* alt_score,
+                 double* best_score, double* second_score, double* alt_score, double* ingroup_gap,
                  int32_t* n_children, uint8_t* status, int n_threads) {
     const Trie& T = *static_cast<const Trie*>(h);
     parallel_rows(n, n_threads, [&](int64_t i) {
@@ -442,6 +494,7 @@ void oracle_step(const void* h, const void* logits, int dtype, int64_t ld, int64
         logq[i] = o.logq; logp[i] = o.logp;
         best_score[i] = o.best; second_score[i] = o.second;
         if (alt_score) alt_score[i] = o.alt;
+        if (ingroup_gap) ingroup_gap[i] = o.ingroup_gap;
         if (n_children) n_children[i] = o.n_children;
         status[i] = o.status;
     });
@@ -522,8 +575,11 @@ void oracle_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* ou
     philox4x32_10(ctr, key, out);
 }
 
-double oracle_gumbel_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t v) {
-    return gumbel_uniform(seed, step, row, v);
+double oracle_group_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t G) {
+    return group_uniform(seed, step, row, G);
+}
+double oracle_ingroup_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t G) {
+    return ingroup_uniform(seed, step, row, G);
 }
 double oracle_resample_uniform(uint64_t seed, uint32_t query) { return resample_uniform(seed, query); }
 double oracle_accept_uniform(uint64_t seed, uint32_t query, uint32_t k) { return accept_uniform(seed, query, k); }

@@ -70,10 +70,20 @@ def test_log_softmax_quantities_match_scipy(dtype, inv_t):
         assert t in A
         np.testing.assert_allclose(o["logq"][i], z[i, t] - lse_ok, atol=1e-12)
         np.testing.assert_allclose(o["logp"][i], z[i, t] - lse_all, atol=1e-12)
-        # the chosen token maximises z + Gumbel noise; noise from the published uniform
-        scores = {v: z[i, v] - np.log(-np.log(oracle.gumbel_uniform(5, 2, i, v))) for v in A}
-        assert t == max(sorted(scores), key=lambda v: scores[v])
-        np.testing.assert_allclose(o["best"][i], scores[t], atol=1e-12)
+        # stage 1: the token's group (8 consecutive ids) maximises log(group mass) + Gumbel noise,
+        # noise from the published uniform; stage 2: inverse CDF inside that group
+        groups = {}
+        for v in A:
+            groups.setdefault(v >> 3, []).append(v)
+        scores = {G: logsumexp(z[i, vs]) - np.log(-np.log(oracle.group_uniform(5, 2, i, G)))
+                  for G, vs in groups.items()}
+        Gw = max(sorted(scores), key=lambda G: scores[G])
+        assert t >> 3 == Gw
+        np.testing.assert_allclose(o["best"][i], scores[Gw], atol=1e-12)
+        vs = groups[Gw]
+        cum = np.cumsum(np.exp(z[i, vs] - z[i, vs].max()))
+        target = oracle.ingroup_uniform(5, 2, i, Gw) * cum[-1]
+        assert t == vs[min(len(vs) - 1, int(np.searchsorted(cum, target, side="right")))]
         # range of the extended prefix and leaf test
         p2 = prefix[i].copy()
         p2[depth[i]] = t
