@@ -31,12 +31,17 @@
  *     bits at positions >= V are zero.
  *   - Random numbers: Philox4x32-10, key = (seed low 32 bits, seed high 32 bits).  The uniform of
  *     output word r is u = ((r >> 9) + 0.5) * 2^-23 (u and 1-u exact in fp32).  Counters:
- *       sampling  (v >> 2, step, row, 0), word v & 3     one uniform per (row, step, token v)
- *       resample  (query, 0, 0, 1), word 0
- *       accept    (query, k, 0, 2), word 0
+ *       group noise  (((G>>10)<<8) | (G&255), step, row, 0), word (G>>8)&3   per token group G
+ *       in-group     (G, step, row, 3), word 0
+ *       resample     (query, 0, 0, 1), word 0
+ *       accept       (query, k, 0, 2), word 0
  *     where `row` / `query` is row_base / query_base plus the index inside the call.
- *   - Sampling is Gumbel-max: token = argmax over allowed v of z_v/T - log(-log u_v), lowest id on
- *     an exact tie; this draws from P.mask/|P.mask|_1.
+ *   - Sampling draws exactly from P.mask/|P.mask|_1 in two stages.  Tokens are taken in groups of
+ *     8 consecutive ids (G = v >> 3).  Stage 1 is Gumbel-max over groups: the group maximising
+ *     log(sum of e^{z_v/T} over its allowed tokens) - log(-log u_G) wins (the lowest G on an exact
+ *     tie); it is therefore chosen with probability proportional to its allowed mass.  Stage 2
+ *     picks, inside the winner, the smallest allowed token whose inclusive cumulative weight
+ *     exceeds u' * mass (tokens in ascending id).
  */
 #ifndef DISC_H_
 #define DISC_H_
@@ -150,11 +155,12 @@ int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
  *   mask_out    device, uint32[n][W] (nullable): the valid-set mask used by each live row
  *   status_out  device, uint8[n]
  * Per live row: z_v = logit_v / T; lse_all = log sum_v e^{z_v}; lse_ok = the same over the valid
- * set; logw += lse_ok - lse_all; token by Gumbel-max over the valid set; the state moves to the
- * extended prefix; done is set when the extended prefix is a member.  Rows with done != 0 are
- * skipped (status DISC_ROW_DONE, token -1, no logits read).  A row whose valid mass is zero keeps
- * going with the lowest valid token (status DISC_ROW_NOMASS, logw = -inf); NaN/+Inf logits give
- * status DISC_ROW_NONFINITE and a NaN/Inf logw. */
+ * set; logw += lse_ok - lse_all; token drawn from the valid set (two-stage rule at the top of this
+ * file); the state moves to the extended prefix; done is set when the extended prefix is a member.
+ * Rows with done != 0 are skipped (status DISC_ROW_DONE, token -1, no logits read).  A row whose
+ * valid mass is zero keeps going with the lowest valid token (status DISC_ROW_NOMASS,
+ * logw = -inf); NaN/+Inf logits give status DISC_ROW_NONFINITE, a NaN/Inf logw and some valid
+ * token (which one is unspecified). */
 int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n,
               float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base,
               int32_t* node, int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done,
@@ -181,9 +187,9 @@ int disc_resample(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_
 int disc_accept(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_t query_base,
                 int32_t* first_out, void* stream);
 
-/* Diagnostic: the n sampling uniforms of tokens v0 .. v0+n-1 for (seed, step, row), as fp32.
+/* Diagnostic: the n group-noise uniforms of token groups g0 .. g0+n-1 for (seed, step, row), fp32.
  *   out  device, float[n] */
-int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t v0, int32_t n,
+int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t g0, int32_t n,
                            float* out, void* stream);
 
 /* Text for a DISC_ERR_* code. */

@@ -1,6 +1,7 @@
 // disc_step: one decoding step of Algorithm 1 (lines 5-8) for a batch of candidates, fused:
-// valid-set lookup, masked and unmasked log-sum-exp over the V logits, Gumbel-max sampling,
-// importance log-weight update and the move of the row's cursor to the extended prefix.
+// valid-set lookup, masked and unmasked log-sum-exp over the V logits, sampling from the masked
+// distribution, importance log-weight update and the move of the row's cursor to the extended
+// prefix.
 //
 // One thread block per row.
 //   * Streaming.  The row's logits are pulled into a shared-memory ring by bulk asynchronous
@@ -8,7 +9,7 @@
 //     flight per block whatever the register budget.  The first chunks are issued before the
 //     block reads the prefix index.  Rows that are not 16-byte aligned take a scalar-load path.
 //   * Sums.  Each thread accumulates sum 2^(x*c - ref) against its own reference (the maximum of
-//     the first vector it sees), c = log2(e)/T.  Per pair of logits: two unpack operations, one
+//     the first logits it sees), c = log2(e)/T.  Per pair of logits: two unpack operations, one
 //     packed fp32x2 FMA, two ex2 and one packed add.  Partial sums are kept as (m, s) pairs meaning
 //     2^m * s and merged exactly.  All differences are formed between references before any large
 //     value is added, so a common offset of the logits does not cost accuracy.
@@ -16,18 +17,23 @@
 //     most DISC_HEAVY_MIN children gather their few logits directly ("gather path").  Rows with
 //     more have a prebuilt bitmask row in global memory; its slice travels into the ring stage next
 //     to the logits it covers ("dense path").
-//   * Sampling.  token = argmax over allowed v of (x_v - xref)/T + g_v with g_v = -log(-log u_v),
-//     u_v from Philox4x32-10 keyed by (token, step, row).  In the dense path a token is evaluated
-//     exactly only if it can still win: with w = 1 - u, g > t implies w < e^-t, so a token whose
-//     w is at least e^(z - best) (times a safety factor) is skipped without taking a logarithm;
-//     e^(z - best) is the already computed 2^(x*c - ref) times a per-thread constant.  `best` is the
-//     best score any lane of the warp has seen (shared once per chunk), which keeps the number of
-//     exact evaluations per warp near log(tokens).
+//   * Sampling (exact draw from P.mask/|P.mask|_1, Algorithm 1 line 7) in two stages.  Stage 1 is
+//     Gumbel-max over groups of 8 consecutive token ids: score_G = log(allowed mass of G) + g_G,
+//     g_G = -log(-log u_G), u_G from Philox4x32-10 keyed by (group, step, row); the best group
+//     wins, the lowest on a tie.  Stage 2 is an inverse-CDF draw among the winner's allowed tokens
+//     with one more uniform.  In the dense path a group is evaluated exactly only if it can still
+//     win: with w = 1 - u, g > t implies w < e^-t, so a group whose w is at least
+//     mass_G / e^best (times a safety factor) is skipped without taking a logarithm; mass_G is
+//     the already accumulated sum of 2^(x*c - ref) times a per-thread constant.  `best` is the
+//     best score any lane of the warp has seen (shared once per chunk).  The four groups a thread
+//     owns in one chunk share one Philox counter.
 //   * A row whose fast sums are not finite, or whose valid mass is so small that terms may have
 //     underflowed against a thread's reference, is redone by a plain two-pass routine with exact
 //     scores ("careful path").
 
 #include <math_constants.h>
+
+#include <type_traits>
 
 #include "disc_internal.cuh"
 
@@ -51,6 +57,7 @@ constexpr int MASK_SLICE_MAX = CHUNK_VECS;               // mask bytes of one st
 constexpr int STAGE_BYTES = CHUNK_BYTES + MASK_SLICE_MAX;
 constexpr int STAGES = DISC_STAGES;
 constexpr int RING_BYTES = STAGE_BYTES * STAGES;
+constexpr int GROUP = 8;                                 // tokens per sampling group
 constexpr uint64_t WAIT_LIMIT_NS = 250ull * 1000 * 1000;  // an mbarrier wait gives up after 0.25 s
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
@@ -95,16 +102,26 @@ __device__ __forceinline__ MS ms_merge(MS a, MS b) {
     return MS{M, a.s * exp2f(a.m - M) + b.s * exp2f(b.m - M)};
 }
 
+// sum of 2^(x*c2) kept as 2^m * s; fma(x, c2, -m) is the exact product minus the reference, so a
+// large common offset of the logits costs no accuracy.  NaN and +inf poison the sum (s = NaN).
+__device__ __forceinline__ void ms_add(MS& a, float x, float c2) {
+    const float y = x * c2;
+    if (!(y < CUDART_INF_F)) a.s = CUDART_NAN_F;
+    else if (y > a.m) { a.s = a.s * exp2f(a.m - y) + exp2f(fmaf(x, c2, -y)); a.m = y; }
+    else if (y != -CUDART_INF_F) a.s += exp2f(fmaf(x, c2, -a.m));
+}
+
 struct Best {
     float score;
-    int32_t tok;     // -1: none yet
-    int32_t child;   // node id of the child when known, else -1
+    int32_t key;     // -1: none yet; dense rows: winning group (token id >> 3); gather rows: the token
+                     // already drawn inside the winning group
+    int32_t child;   // gather rows: index node of that token, else -1
 };
 
 __device__ __forceinline__ Best best_merge(Best a, Best b) {
-    if (b.tok < 0) return a;
-    if (a.tok < 0) return b;
-    if (b.score > a.score || (b.score == a.score && b.tok < a.tok)) return b;
+    if (b.key < 0) return a;
+    if (a.key < 0) return b;
+    if (b.score > a.score || (b.score == a.score && b.key < a.key)) return b;
     return a;
 }
 
@@ -168,7 +185,7 @@ struct Elem<DISC_F32> {
     __device__ static __forceinline__ float load(const void* base, int64_t i) {
         return __ldg(static_cast<const float*>(base) + i);
     }
-    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&x)[2]) {
+    __device__ static __forceinline__ void unpack(const uint4& v, float2* x) {
         x[0] = make_float2(__uint_as_float(v.x), __uint_as_float(v.y));
         x[1] = make_float2(__uint_as_float(v.z), __uint_as_float(v.w));
     }
@@ -183,18 +200,21 @@ struct Elem<DISC_BF16> {
     __device__ static __forceinline__ float2 pair(uint32_t w) {
         return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
     }
-    __device__ static __forceinline__ void unpack(const uint4& v, float2 (&x)[4]) {
+    __device__ static __forceinline__ void unpack(const uint4& v, float2* x) {
         x[0] = pair(v.x); x[1] = pair(v.y); x[2] = pair(v.z); x[3] = pair(v.w);
     }
 };
 
-// Gumbel-perturbed score of a token with raw logit x, relative to the row's reference logit xref.
-// The argmax does not depend on the common shift, and subtracting before scaling keeps the score
-// accurate to a few ulp of (x - xref) whatever offset the logits carry.  Kept out of line: it is
-// reached for a handful of tokens per warp and row, and inlining it at every call site would
-// multiply the size of the streaming loop.
-__device__ __noinline__ float gumbel_score(float x, float xref, float inv_t, uint32_t word) {
-    return (x - xref) * inv_t + gumbel_from_uniform(uniform_from_bits(word));
+// ---- sampling helpers ---------------------------------------------------------------------------
+// Philox counter word 0 and output word of group G.  The four groups a thread owns in one ring
+// chunk (256 apart) share a counter.
+__device__ __forceinline__ uint32_t group_slot(uint32_t G) { return ((G >> 10) << 8) | (G & 255u); }
+__device__ __forceinline__ uint32_t group_word(uint32_t G) { return (G >> 8) & 3u; }
+
+// Exact score of a group whose allowed mass is 2^mlog2 (relative to the row's reference logit):
+// ln(mass) + Gumbel noise.  Kept out of line: it runs for a handful of groups per warp and row.
+__device__ __noinline__ float group_score(float mlog2, uint32_t word) {
+    return mlog2 * LN2_F + gumbel_from_uniform(uniform_from_bits(word));
 }
 
 // w = 1 - u of a random word, exact: with k' the complement of the word's top 23 bits,
@@ -203,8 +223,8 @@ __device__ __forceinline__ float complement_uniform(uint32_t word) {
     return __uint_as_float(0x3f800000u | ((~word) >> 9)) - 0.99999994039535522f;
 }
 
-__device__ __forceinline__ bool mask_bit(const uint32_t* __restrict__ gmask, int v) {
-    return (__ldg(gmask + (v >> 5)) >> (v & 31)) & 1u;
+__device__ __forceinline__ uint32_t mask_byte(const uint32_t* __restrict__ gmask, uint32_t G) {
+    return (__ldg(gmask + (G >> 2)) >> ((G & 3u) * 8u)) & 0xFFu;
 }
 
 // Per-thread accumulators of the streaming loop.
@@ -216,8 +236,8 @@ struct Acc {
     // sampling
     Best best{-__builtin_huge_valf(), -1, -1};
     float bound_best = -__builtin_huge_valf();   // best score known to this warp (>= best.score)
-    float cbase = 0.f;                            // mref - xref*c
-    float cbound = __builtin_huge_valf();   // SAFETY * 2^(cbase - bound_best*log2e): e*cbound >= e^(z-best)
+    float cbase = 0.f;                            // mref - xref*c: log2 of (thread sums -> row-relative mass)
+    float cbound = __builtin_huge_valf();   // SAFETY * 2^(cbase - bound_best*log2e): t*cbound >= mass/e^best
 };
 
 struct RowCtx {
@@ -237,13 +257,19 @@ __device__ __forceinline__ void set_reference(Acc& a, const RowCtx& r, float xma
     update_bound(a);
 }
 
-__device__ __forceinline__ void exact_candidate(Acc& a, const RowCtx& r, float x, uint32_t word, int32_t v) {
-    // Tokens arrive in ascending order inside a thread, so strict '>' keeps the lowest id on a
+// exact evaluation of group G whose allowed terms sum to t (against this thread's reference)
+__device__ __forceinline__ void exact_group(Acc& a, float t, uint32_t word, int32_t G) {
+    // Groups arrive in ascending order inside a thread, so strict '>' keeps the lowest group on a
     // tie.  NaN and -inf scores never win; a row without any finite score falls back to its
     // lowest valid token at the end.
-    const float score = gumbel_score(x, r.xref, r.inv_t, word);
-    if (score > a.best.score) { a.best.score = score; a.best.tok = v; a.best.child = -1; }
+    const float score = group_score(a.cbase + log2f(t), word);
+    if (score > a.best.score) { a.best.score = score; a.best.key = G; a.best.child = -1; }
     if (score > a.bound_best) { a.bound_best = score; update_bound(a); }
+}
+
+// skip test + exact evaluation of one group
+__device__ __forceinline__ void sample_group(Acc& a, float t, uint32_t word, int32_t G) {
+    if (!(complement_uniform(word) >= t * a.cbound)) exact_group(a, t, word, G);
 }
 
 // share the best score of the warp's lanes (called at warp-uniform points)
@@ -255,38 +281,12 @@ __device__ __forceinline__ void share_bound(Acc& a) {
     update_bound(a);
 }
 
-// the four tokens 4g .. 4g+3 of one Philox counter; nib = which of them are allowed
-__device__ __forceinline__ void sample_group(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, uint32_t g,
-                                             uint32_t nib, float x0, float x1, float x2, float x3, float e0,
-                                             float e1, float e2, float e3) {
-    // No token of this group can win if even the largest noise is not enough: w >= 2^-24 always,
-    // so e*cbound < 2^-24 for all four means "skip" without drawing the random numbers.
-#ifdef DISC_EXP_NOSAMPLE
-    return;
-#endif
-    const float emax = fmaxf(fmaxf(e0, e1), fmaxf(e2, e3));
-    if (emax * a.cbound < TWO_M24) return;
-#ifdef DISC_EXP_CHEAPRNG
-    const uint32_t hh = (g * 2654435761u) ^ (r.row * 40503u) ^ rk.k[0];
-    const uint4 w4 = make_uint4(hh, hh * 3u, hh * 5u, hh * 7u);
-#else
-    const uint4 w4 = philox4x32_10(g, r.step, r.row, 0u, rk);
-#endif
-    const int32_t v = int32_t(g << 2);
-    if ((nib & 1u) && !(complement_uniform(w4.x) >= e0 * a.cbound)) exact_candidate(a, r, x0, w4.x, v);
-    if ((nib & 2u) && !(complement_uniform(w4.y) >= e1 * a.cbound)) exact_candidate(a, r, x1, w4.y, v + 1);
-    if ((nib & 4u) && !(complement_uniform(w4.z) >= e2 * a.cbound)) exact_candidate(a, r, x2, w4.z, v + 2);
-    if ((nib & 8u) && !(complement_uniform(w4.w) >= e3 * a.cbound)) exact_candidate(a, r, x3, w4.w, v + 3);
-}
-
-// one 16-byte vector of logits starting at token v0 (a multiple of the vector width);
-// bits = allowed flags of its EPV tokens (dense path only)
-template <int DT, bool DENSE>
-__device__ __forceinline__ void consume_vec(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const uint4& raw,
-                                            int v0, uint32_t bits) {
+// exponentials of one 16-byte vector; returns their pairwise sum in t
+template <int DT>
+__device__ __forceinline__ float2 vec_exp(const Acc& a, const RowCtx& r, const uint4& raw, float2* e) {
     using E = Elem<DT>;
     constexpr int NP = E::EPV / 2;
-    float2 x[NP], e[NP];
+    float2 x[NP];
     E::unpack(raw, x);
     const float2 cc = make_float2(r.c2, r.c2), nm = make_float2(-a.mref, -a.mref);
 #pragma unroll
@@ -294,51 +294,63 @@ __device__ __forceinline__ void consume_vec(Acc& a, const RowCtx& r, const Philo
         const float2 y = __ffma2_rn(x[i], cc, nm);
         e[i] = make_float2(ex2_approx(y.x), ex2_approx(y.y));
     }
-    if constexpr (!DENSE) {
+    float2 t = __fadd2_rn(e[0], e[1]);
+    if constexpr (NP == 4) t = __fadd2_rn(t, __fadd2_rn(e[2], e[3]));
+    return t;
+}
+
+// sparse rows: one 16-byte vector of logits
+template <int DT>
+__device__ __forceinline__ void consume_vec_sparse(Acc& a, const RowCtx& r, const uint4& raw) {
+    using E = Elem<DT>;
+    constexpr int NP = E::EPV / 2;
+    float2 x[NP];
+    E::unpack(raw, x);
+    const float2 cc = make_float2(r.c2, r.c2), nm = make_float2(-a.mref, -a.mref);
 #pragma unroll
-        for (int i = 0; i < NP; i += 2) {
-            a.sa = __fadd2_rn(a.sa, e[i]);
-            a.sb = __fadd2_rn(a.sb, e[i + 1]);
-        }
-    } else {
-        float2 t = __fadd2_rn(e[0], e[1]);
-        if constexpr (NP == 4) t = __fadd2_rn(t, __fadd2_rn(e[2], e[3]));
-        a.sa = __fadd2_rn(a.sa, t);
-        constexpr uint32_t FULL = (1u << E::EPV) - 1u;
-        if (bits) {
-            if (bits == FULL) {
-                a.ok2 = __fadd2_rn(a.ok2, t);
-            } else {
-#pragma unroll
-                for (int i = 0; i < NP; ++i) {
-                    a.ok2.x += ((bits >> (2 * i)) & 1u) ? e[i].x : 0.f;
-                    a.ok2.y += ((bits >> (2 * i + 1)) & 1u) ? e[i].y : 0.f;
-                }
-            }
-#pragma unroll
-            for (int q = 0; q < NP / 2; ++q) {
-                const uint32_t nib = (bits >> (4 * q)) & 0xFu;
-                if (nib)
-                    sample_group(a, r, rk, uint32_t(v0 >> 2) + q, nib, x[2 * q].x, x[2 * q].y, x[2 * q + 1].x,
-                                 x[2 * q + 1].y, e[2 * q].x, e[2 * q].y, e[2 * q + 1].x, e[2 * q + 1].y);
-            }
-        }
+    for (int i = 0; i < NP; i += 2) {
+        const float2 y0 = __ffma2_rn(x[i], cc, nm), y1 = __ffma2_rn(x[i + 1], cc, nm);
+        a.sa = __fadd2_rn(a.sa, make_float2(ex2_approx(y0.x), ex2_approx(y0.y)));
+        a.sb = __fadd2_rn(a.sb, make_float2(ex2_approx(y1.x), ex2_approx(y1.y)));
     }
 }
 
-// one logit (scalar path and ragged tail); the allowed flag comes from the global mask row
+// dense rows: the allowed part of one vector's exponentials; nb = allowed flags of its tokens
+template <int NP>
+__device__ __forceinline__ float masked_sum(const float2* e, const float2& t, uint32_t nb) {
+    constexpr uint32_t FULL = (1u << (2 * NP)) - 1u;
+    if (nb == FULL) return t.x + t.y;
+    float s0 = 0.f, s1 = 0.f;
+    if (nb) {
+#pragma unroll
+        for (int i = 0; i < NP; ++i) {
+            s0 += ((nb >> (2 * i)) & 1u) ? e[i].x : 0.f;
+            s1 += ((nb >> (2 * i + 1)) & 1u) ? e[i].y : 0.f;
+        }
+    }
+    return s0 + s1;
+}
+
+// one group given as up to 8 scalars (scalar path, ragged tails, careful use): x[j] for j < nvalid
 template <bool DENSE>
-__device__ __forceinline__ void consume_one(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, float x, int v,
-                                            const uint32_t* __restrict__ gmask) {
-    if (!a.touched) set_reference(a, r, x);
-    const float e = ex2_approx(fmaf(x, r.c2, -a.mref));
-    a.sa.x += e;
-    if (DENSE && mask_bit(gmask, v)) {
-        a.ok2.x += e;
-        if (!(e * a.cbound < TWO_M24)) {
-            const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, rk);
-            const uint32_t word = pick_word(w4, v & 3);
-            if (!(complement_uniform(word) >= e * a.cbound)) exact_candidate(a, r, x, word, v);
+__device__ __forceinline__ void consume_group_scalar(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk,
+                                                     const float* x, int nvalid, uint32_t G, uint32_t bits) {
+    if (!a.touched) {
+        float mx = x[0];
+        for (int j = 1; j < nvalid; ++j) mx = fmaxf(mx, x[j]);
+        set_reference(a, r, mx);
+    }
+    float t = 0.f;
+    for (int j = 0; j < nvalid; ++j) {
+        const float e = ex2_approx(fmaf(x[j], r.c2, -a.mref));
+        a.sa.x += e;
+        if (DENSE && ((bits >> j) & 1u)) t += e;
+    }
+    if (DENSE && bits) {
+        a.ok2.x += t;
+        if (!(t * a.cbound < TWO_M24)) {
+            const uint4 w4 = philox4x32_10(group_slot(G), r.step, r.row, 0u, rk);
+            sample_group(a, t, pick_word(w4, group_word(G)), int32_t(G));
         }
     }
 }
@@ -400,7 +412,7 @@ __device__ int32_t warp_find_child(const int32_t* __restrict__ node_tok, int32_t
 struct RingGeom {
     const char* rowp;        // the row's logits
     const char* gmask;       // the row's prebuilt mask (dense rows), else nullptr
-    uint32_t vec_bytes;      // bytes of whole 16-byte vectors in the row
+    uint32_t vec_bytes;      // bytes of the row that go through the ring (whole groups of 8 tokens)
     uint32_t mask_bytes;     // bytes of the mask row that may be read (a multiple of 16)
     uint32_t slice;          // mask bytes per full chunk
     uint32_t ring_s, full_s; // shared-memory addresses of the ring and of the full barriers
@@ -428,13 +440,23 @@ __device__ __forceinline__ void ring_issue(const RingGeom& g, int c, int s, bool
 // their mask slices right after it, on a barrier of their own (mask0).  Then thread 0 keeps
 // STAGES-1 chunks in flight: after every warp has copied chunk c-1 out of its stage (empty
 // barrier), that stage is refilled with chunk c-1+STAGES.  Returns false if a wait gave up.
+//
+// Work split inside a chunk.  Sparse rows: thread t takes vectors t, t+256, t+512, t+768.  Dense
+// rows work on groups of 8 tokens: bf16 - the same four vectors (one group each); f32 - groups t
+// and t+256 of the chunk's 512 (two adjacent vectors each).  Either way the groups of one thread
+// in one chunk are 256 apart and share a Philox counter.
 template <int DT, bool DENSE>
 __device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const RingGeom& g, int V,
                             const unsigned char* ring, uint32_t empty_s, uint32_t mask0_s) {
     using E = Elem<DT>;
     constexpr int EPV = E::EPV;
+    constexpr int NP = EPV / 2;
+    constexpr int VPG = GROUP / EPV;                          // vectors per group: 1 (bf16) or 2 (f32)
+    constexpr int GPT = VPT / VPG;                            // groups per thread and chunk
+    constexpr int GPC = GPT * STEP_THREADS;                   // groups per chunk
     const int tid = threadIdx.x, lane = tid & 31;
-    const int nvec = V / EPV;
+    const int nvec = int(g.vec_bytes / 16u);
+    const int ngroups = nvec / VPG;
     const int n_chunks = int((g.vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
     const int n_full = int(g.vec_bytes / CHUNK_BYTES);
     bool ok = true;
@@ -451,55 +473,101 @@ __device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, 
         if (!__all_sync(0xffffffffu, mbar_wait(g.full_s + 8u * s, ph))) { ok = false; break; }
         const unsigned char* stage_b = ring + s * STAGE_BYTES;
         const uint4* stage = reinterpret_cast<const uint4*>(stage_b);
-        uint4 raw[VPT];
-        uint32_t bits[VPT];
-        const bool full = c < n_full;
-        const int g0 = c * CHUNK_VECS + tid;
+
+        auto body = [&](auto full_tag) {
+            constexpr bool FULL = decltype(full_tag)::value;
+            uint4 raw[VPT];
+            uint32_t bits[GPT];
+            bool have[VPT];
+            // vector index inside the chunk of this thread's k-th vector
+            auto vidx = [&](int k) { return DENSE ? ((k / VPG) * STEP_THREADS + tid) * VPG + (k % VPG)
+                                                  : k * STEP_THREADS + tid; };
 #pragma unroll
-        for (int j = 0; j < VPT; ++j) {
-            bits[j] = 0;
-            if (full || g0 + j * STEP_THREADS < nvec) {
-                raw[j] = stage[j * STEP_THREADS + tid];
-                if constexpr (DENSE) {
-                    const int iv = j * STEP_THREADS + tid;       // vector index inside the chunk
-                    if constexpr (EPV == 8) bits[j] = stage_b[CHUNK_BYTES + iv];
-                    else bits[j] = (uint32_t(stage_b[CHUNK_BYTES + (iv >> 1)]) >> ((iv & 1) * 4)) & 0xFu;
+            for (int k = 0; k < VPT; ++k) {
+                have[k] = FULL || (c * CHUNK_VECS + vidx(k) < nvec);
+                if (have[k]) raw[k] = stage[vidx(k)];
+            }
+            if constexpr (DENSE) {
+#pragma unroll
+                for (int j = 0; j < GPT; ++j) {
+                    const int gi = j * STEP_THREADS + tid;           // group index inside the chunk
+                    bits[j] = (FULL || c * GPC + gi < ngroups) ? uint32_t(stage_b[CHUNK_BYTES + gi]) : 0u;
                 }
             }
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(empty_s + 8u * s);
-        if (tid == 0 && c >= 1 && c - 1 + STAGES < n_chunks) {
-            if (!mbar_wait(empty_s + 8u * sp, php)) ok = false;
-            else ring_issue(g, c - 1 + STAGES, sp, DENSE);
-        }
-        if (c == 0 && tid < nvec) {
-            float2 x[EPV / 2];
-            E::unpack(raw[0], x);
-            float mx = fmaxf(x[0].x, x[0].y);
+            __syncwarp();
+            if (lane == 0) mbar_arrive(empty_s + 8u * s);
+            if (tid == 0 && c >= 1 && c - 1 + STAGES < n_chunks) {
+                if (!mbar_wait(empty_s + 8u * sp, php)) ok = false;
+                else ring_issue(g, c - 1 + STAGES, sp, DENSE);
+            }
+            if (c == 0 && have[0]) {
+                float2 x[NP];
+                E::unpack(raw[0], x);
+                float mx = fmaxf(x[0].x, x[0].y);
 #pragma unroll
-            for (int i = 1; i < EPV / 2; ++i) mx = fmaxf(mx, fmaxf(x[i].x, x[i].y));
-            set_reference(a, r, mx);
-        }
+                for (int i = 1; i < NP; ++i) mx = fmaxf(mx, fmaxf(x[i].x, x[i].y));
+                set_reference(a, r, mx);
+            }
+            if constexpr (!DENSE) {
 #pragma unroll
-        for (int j = 0; j < VPT; ++j)
-            if (full || g0 + j * STEP_THREADS < nvec)
-                consume_vec<DT, DENSE>(a, r, rk, raw[j], (g0 + j * STEP_THREADS) * EPV, bits[j]);
-        if constexpr (DENSE) share_bound(a);
+                for (int k = 0; k < VPT; ++k)
+                    if (have[k]) consume_vec_sparse<DT>(a, r, raw[k]);
+            } else {
+                float tg[GPT];
+#pragma unroll
+                for (int j = 0; j < GPT; ++j) {
+                    tg[j] = 0.f;
+#pragma unroll
+                    for (int h = 0; h < VPG; ++h) {
+                        const int k = j * VPG + h;
+                        if (have[k]) {
+                            float2 e[NP];
+                            const float2 t = vec_exp<DT>(a, r, raw[k], e);
+                            a.sa = __fadd2_rn(a.sa, t);
+                            tg[j] += masked_sum<NP>(e, t, (bits[j] >> (h * EPV)) & ((1u << EPV) - 1u));
+                        }
+                    }
+                    a.ok2.x += tg[j];
+                }
+                // stage 1 of the sampling for this thread's groups of the chunk: nothing to do if
+                // even the largest possible noise cannot lift any of them above the best score
+                float tmax = tg[0];
+#pragma unroll
+                for (int j = 1; j < GPT; ++j) tmax = fmaxf(tmax, tg[j]);
+                if (!(tmax * a.cbound < TWO_M24)) {
+                    const uint32_t G0 = uint32_t(c * GPC + tid);
+                    const uint4 w4 = philox4x32_10(group_slot(G0), r.step, r.row, 0u, rk);
+#pragma unroll
+                    for (int j = 0; j < GPT; ++j) {
+                        const uint32_t G = G0 + uint32_t(j * STEP_THREADS);
+                        if (bits[j]) sample_group(a, tg[j], pick_word(w4, group_word(G)), int32_t(G));
+                    }
+                }
+                share_bound(a);
+            }
+        };
+        if (c < n_full) body(std::true_type{}); else body(std::false_type{});
+
         sp = s; php = ph;
         if (++s == STAGES) { s = 0; ph ^= 1u; }
     }
-    // ragged tail: V not a multiple of the vector width
-    const int v = nvec * EPV + tid;
-    if (v < V) consume_one<DENSE>(a, r, rk, E::load(g.rowp, v), v, reinterpret_cast<const uint32_t*>(g.gmask));
     return ok;
 }
 
+// groups [g_begin, g_end) of the row read with scalar loads (whole row on the scalar path; the
+// ragged last group on the ring path)
 template <int DT, bool DENSE>
-__device__ void stream_scalar(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp, int V,
-                              const uint32_t* gmask) {
+__device__ void stream_groups_scalar(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp, int V,
+                                     const uint32_t* gmask, int g_begin, int g_end) {
     using E = Elem<DT>;
-    for (int v = threadIdx.x; v < V; v += STEP_THREADS) consume_one<DENSE>(a, r, rk, E::load(rowp, v), v, gmask);
+    for (int G = g_begin + threadIdx.x; G < g_end; G += STEP_THREADS) {
+        float x[GROUP];
+        const int v0 = G * GROUP;
+        const int nvalid = min(GROUP, V - v0);
+        for (int j = 0; j < nvalid; ++j) x[j] = E::load(rowp, v0 + j);
+        const uint32_t bits = DENSE ? mask_byte(gmask, uint32_t(G)) : 0u;
+        consume_group_scalar<DENSE>(a, r, rk, x, nvalid, uint32_t(G), bits);
+    }
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
@@ -525,13 +593,15 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_DONE; }
         return;
     }
-    // Start streaming before anything else: the first ring stage fills while the index is read.
+    // Start streaming before anything else: the first ring stages fill while the index is read.
+    const int n_groups = (p.V + GROUP - 1) / GROUP;       // the last one may be ragged
+    const int n_ring_groups = RING ? p.V / GROUP : 0;     // whole groups go through the ring
     RingGeom g;
     g.rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
     g.gmask = nullptr;
-    g.vec_bytes = uint32_t(p.V / E::EPV) * 16u;
+    g.vec_bytes = uint32_t(n_ring_groups) * uint32_t(GROUP * E::SIZE);
     g.mask_bytes = uint32_t(p.Wp) * 4u;
-    g.slice = uint32_t(CHUNK_VECS * E::EPV / 8);
+    g.slice = uint32_t(CHUNK_VECS * E::EPV / GROUP);
     g.ring_s = smem_u32(ring);
     g.full_s = smem_u32(full_bar);
     const int n_chunks = int((g.vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
@@ -600,7 +670,6 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 
     Acc a;
     MS ok{-CUDART_INF_F, 0.f};
-    bool poisoned = false;
 
     if (p.mask_out) {
         // optional output of the valid-set mask
@@ -617,19 +686,60 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         }
     }
     if (!dense) {
-        // gather path: the few allowed logits are read directly
+        // gather path: the few allowed logits are read directly.  Every thread adds its child to
+        // the valid-set sum; the thread holding the first child of a group also collects the
+        // group's members (at most 8 children), forms the group's exact score and, if that score
+        // is the best it has seen, draws the token inside the group right away (stage 2), so that
+        // nothing of this is left for the end of the block.
         for (int i = tid; i < c; i += STEP_THREADS) {
             const int32_t v = __ldg(p.node_tok + cb + i);
             const float x = E::load(g.rowp, v);
-            // sum of 2^(x*c2) kept as 2^m * s; fma(x, c2, -m) is the exact product minus the
-            // reference, so a large common offset of the logits costs no accuracy
-            const float y = x * p.c2;
-            if (!(y < CUDART_INF_F)) poisoned = true;                 // NaN or +inf: careful path
-            else if (y > ok.m) { ok.s = ok.s * exp2f(ok.m - y) + exp2f(fmaf(x, p.c2, -y)); ok.m = y; }
-            else if (y != -CUDART_INF_F) ok.s += exp2f(fmaf(x, p.c2, -ok.m));
-            const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, p.rk);
-            const float score = gumbel_score(x, r.xref, r.inv_t, pick_word(w4, v & 3));
-            if (score > a.best.score) { a.best.score = score; a.best.tok = v; a.best.child = cb + i; }
+            ms_add(ok, x, p.c2);
+            const int32_t G = v >> 3;
+            const bool leader = (i == 0) || ((__ldg(p.node_tok + cb + i - 1) >> 3) != G);
+            if (leader) {
+                float xs[GROUP];
+                xs[0] = x;
+                int n = 1;
+#pragma unroll
+                for (int k = 1; k < GROUP; ++k) {
+                    if (n == k && i + k < c) {
+                        const int32_t v2 = __ldg(p.node_tok + cb + i + k);
+                        if ((v2 >> 3) == G) { xs[k] = E::load(g.rowp, v2); n = k + 1; }
+                    }
+                }
+                MS gm{-CUDART_INF_F, 0.f};
+#pragma unroll
+                for (int k = 0; k < GROUP; ++k)
+                    if (k < n) ms_add(gm, xs[k], p.c2);
+                const uint4 w4 = philox4x32_10(group_slot(uint32_t(G)), r.step, r.row, 0u, p.rk);
+                const float score = group_score(fmaf(-r.xref, p.c2, gm.m) + log2f(gm.s),
+                                                pick_word(w4, group_word(uint32_t(G))));
+                if (score > a.best.score) {
+                    int pick = 0;
+                    if (n > 1) {
+                        // inverse CDF over the members' weights 2^(x*c2 - gm.m), ascending token id
+                        float cum[GROUP];
+                        float total = 0.f;
+#pragma unroll
+                        for (int k = 0; k < GROUP; ++k) {
+                            if (k < n) total += exp2f(fmaf(xs[k], p.c2, -gm.m));
+                            cum[k] = total;
+                        }
+                        if (total > 0.f && total < CUDART_INF_F) {
+                            const uint4 u4 = philox4x32_10(uint32_t(G), r.step, r.row, 3u, p.rk);
+                            const float target = uniform_from_bits(u4.x) * total;
+                            pick = n - 1;
+#pragma unroll
+                            for (int k = GROUP - 2; k >= 0; --k)
+                                if (k < n && cum[k] > target) pick = k;
+                        }
+                    }
+                    a.best.score = score;
+                    a.best.key = __ldg(p.node_tok + cb + i + pick);
+                    a.best.child = cb + i + pick;
+                }
+            }
         }
     }
 
@@ -638,15 +748,13 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     if (RING) {
         waits_ok = dense ? stream_ring<DT, true>(a, r, p.rk, g, p.V, ring, smem_u32(empty_bar), smem_u32(&mask0_bar))
                          : stream_ring<DT, false>(a, r, p.rk, g, p.V, ring, smem_u32(empty_bar), smem_u32(&mask0_bar));
-    } else {
-        if (dense) stream_scalar<DT, true>(a, r, p.rk, g.rowp, p.V, gmask);
-        else stream_scalar<DT, false>(a, r, p.rk, g.rowp, p.V, gmask);
     }
+    if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, g.rowp, p.V, gmask, n_ring_groups, n_groups);
+    else stream_groups_scalar<DT, false>(a, r, p.rk, g.rowp, p.V, gmask, n_ring_groups, n_groups);
     if (!waits_ok) s_fault = 1;
 
     MS all = a.touched ? MS{a.mref, (a.sa.x + a.sa.y) + (a.sb.x + a.sb.y)} : MS{-CUDART_INF_F, 0.f};
     if (dense) ok = a.touched ? MS{a.mref, a.ok2.x + a.ok2.y} : MS{-CUDART_INF_F, 0.f};
-    if (poisoned) ok.s = CUDART_NAN_F;
     Best best = a.best;
 
     __syncthreads();
@@ -663,7 +771,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     for (int o = 16; o > 0; o >>= 1) {
         MS a2{__shfl_xor_sync(0xffffffffu, all.m, o), __shfl_xor_sync(0xffffffffu, all.s, o)};
         MS k2{__shfl_xor_sync(0xffffffffu, ok.m, o), __shfl_xor_sync(0xffffffffu, ok.s, o)};
-        Best b2{__shfl_xor_sync(0xffffffffu, best.score, o), __shfl_xor_sync(0xffffffffu, best.tok, o),
+        Best b2{__shfl_xor_sync(0xffffffffu, best.score, o), __shfl_xor_sync(0xffffffffu, best.key, o),
                 __shfl_xor_sync(0xffffffffu, best.child, o)};
         all = ms_merge(all, a2);
         ok = ms_merge(ok, k2);
@@ -671,7 +779,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     }
     if (lane == 0) {
         red_f[0][warp] = all.m; red_f[1][warp] = all.s; red_f[2][warp] = ok.m; red_f[3][warp] = ok.s;
-        red_f[4][warp] = best.score; red_i[0][warp] = best.tok; red_i[1][warp] = best.child;
+        red_f[4][warp] = best.score; red_i[0][warp] = best.key; red_i[1][warp] = best.child;
     }
     __syncthreads();
     if (warp == 0) {
@@ -688,7 +796,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         for (int o = STEP_WARPS / 2; o > 0; o >>= 1) {
             MS a2{__shfl_xor_sync(0xffffffffu, all.m, o), __shfl_xor_sync(0xffffffffu, all.s, o)};
             MS k2{__shfl_xor_sync(0xffffffffu, ok.m, o), __shfl_xor_sync(0xffffffffu, ok.s, o)};
-            Best b2{__shfl_xor_sync(0xffffffffu, best.score, o), __shfl_xor_sync(0xffffffffu, best.tok, o),
+            Best b2{__shfl_xor_sync(0xffffffffu, best.score, o), __shfl_xor_sync(0xffffffffu, best.key, o),
                     __shfl_xor_sync(0xffffffffu, best.child, o)};
             all = ms_merge(all, a2);
             ok = ms_merge(ok, k2);
@@ -702,33 +810,31 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         const float l2_ok = ok.m + log2f(ok.s);
         // The fast sums are trusted when both are finite.  In the dense path the valid-set sum
         // shares each thread's reference with the full sum, so an allowed term 2^-126 below a
-        // thread's reference is flushed to zero (and its token skipped by the bound).  all.m is the
-        // largest reference; while log2(valid mass) >= all.m - 60 every flushed term is below
-        // 2^-49 of the valid sum even if all 2^17 of them were flushed, and no flushed token can
-        // win (its score trails the best allowed token by more than the largest noise).
+        // thread's reference is flushed to zero (and its group may be skipped by the bound).
+        // all.m is the largest reference; while log2(valid mass) >= all.m - 60 every flushed term
+        // is below 2^-49 of the valid sum even if all 2^17 of them were flushed, and no group made
+        // of flushed terms can win (its score trails the best group by more than the largest noise).
         bool trust = fabsf(l2_all) < CUDART_INF_F && fabsf(l2_ok) < CUDART_INF_F;
         if (dense && !(l2_ok >= all.m - MASS_FLOOR_LOG2)) trust = false;
         s_flag = trust ? 0 : 1;
-        red_f[4][0] = best.score; red_i[0][0] = best.tok; red_i[1][0] = best.child;
+        red_f[4][0] = best.score; red_i[0][0] = best.key; red_i[1][0] = best.child;
     }
     __syncthreads();
 
     if (s_flag) {
         // ---- careful path: plain two-pass log-sum-exp with separate maxima for the full row and
-        // for the valid set.  Dense rows test the prebuilt mask and evaluate the score of every
-        // allowed token exactly again; gather rows walk their child list (their scores were exact).
+        // for the valid set, group by group.  Dense rows test the prebuilt mask and evaluate the
+        // score of every group exactly again; gather rows walk their child list (their group
+        // scores were exact already).
         float mx_all = -CUDART_INF_F, mx_ok = -CUDART_INF_F;
         int nan_all = 0, nan_ok = 0;
-        Best cbest{-CUDART_INF_F, -1, -1};
-        for (int v = tid; v < p.V; v += STEP_THREADS) {
-            const float x = E::load(g.rowp, v);
-            const bool allowed = dense && mask_bit(gmask, v);
-            if (x != x) { nan_all = 1; nan_ok |= allowed; }
-            else { mx_all = fmaxf(mx_all, x); if (allowed) mx_ok = fmaxf(mx_ok, x); }
-            if (allowed) {
-                const uint4 w4 = philox4x32_10(uint32_t(v) >> 2, r.step, r.row, 0u, p.rk);
-                const float score = gumbel_score(x, r.xref, r.inv_t, pick_word(w4, v & 3));
-                if (score > cbest.score) { cbest.score = score; cbest.tok = v; }
+        for (int G = tid; G < n_groups; G += STEP_THREADS) {
+            const uint32_t bits = dense ? mask_byte(gmask, uint32_t(G)) : 0u;
+            for (int j = 0; j < GROUP && G * GROUP + j < p.V; ++j) {
+                const float x = E::load(g.rowp, G * GROUP + j);
+                const bool allowed = (bits >> j) & 1u;
+                if (x != x) { nan_all = 1; nan_ok |= allowed; }
+                else { mx_all = fmaxf(mx_all, x); if (allowed) mx_ok = fmaxf(mx_ok, x); }
             }
         }
         if (!dense) {
@@ -744,10 +850,22 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         const bool fin_all = fabsf(mx_all) < CUDART_INF_F, fin_ok = fabsf(mx_ok) < CUDART_INF_F;
         const float r_all = mx_all * p.c2, r_ok = mx_ok * p.c2;
         float sum_all = 0.f, sum_ok = 0.f;
-        for (int v = tid; v < p.V; v += STEP_THREADS) {
-            const float x = E::load(g.rowp, v);
-            if (fin_all) sum_all += exp2f(fmaf(x, p.c2, -r_all));
-            if (fin_ok && dense && mask_bit(gmask, v)) sum_ok += exp2f(fmaf(x, p.c2, -r_ok));
+        Best cbest{-CUDART_INF_F, -1, -1};
+        for (int G = tid; G < n_groups; G += STEP_THREADS) {
+            const uint32_t bits = dense ? mask_byte(gmask, uint32_t(G)) : 0u;
+            float tg = 0.f;
+            for (int j = 0; j < GROUP && G * GROUP + j < p.V; ++j) {
+                const float x = E::load(g.rowp, G * GROUP + j);
+                if (fin_all) sum_all += exp2f(fmaf(x, p.c2, -r_all));
+                if (fin_ok && ((bits >> j) & 1u)) tg += exp2f(fmaf(x, p.c2, -r_ok));
+            }
+            if (bits && fin_ok) {
+                sum_ok += tg;
+                const uint4 w4 = philox4x32_10(group_slot(uint32_t(G)), r.step, r.row, 0u, p.rk);
+                const float score = group_score(fmaf(-r.xref, p.c2, r_ok) + log2f(tg),
+                                                pick_word(w4, group_word(uint32_t(G))));
+                if (score > cbest.score) { cbest.score = score; cbest.key = G; }
+            }
         }
         if (!dense && fin_ok) {
             for (int i = tid; i < c; i += STEP_THREADS)
@@ -758,16 +876,16 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         if (dense) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) {
-                Best b2{__shfl_xor_sync(0xffffffffu, cbest.score, o), __shfl_xor_sync(0xffffffffu, cbest.tok, o), -1};
+                Best b2{__shfl_xor_sync(0xffffffffu, cbest.score, o), __shfl_xor_sync(0xffffffffu, cbest.key, o), -1};
                 cbest = best_merge(cbest, b2);
             }
             __syncthreads();
-            if (lane == 0) { red_f[5][warp] = cbest.score; red_i[0][warp] = cbest.tok; }
+            if (lane == 0) { red_f[5][warp] = cbest.score; red_i[0][warp] = cbest.key; }
             __syncthreads();
             if (tid == 0) {
                 Best b{red_f[5][0], red_i[0][0], -1};
                 for (int w = 1; w < STEP_WARPS; ++w) b = best_merge(b, Best{red_f[5][w], red_i[0][w], -1});
-                red_f[4][0] = b.score; red_i[0][0] = b.tok; red_i[1][0] = -1;
+                red_f[4][0] = b.score; red_i[0][0] = b.key; red_i[1][0] = -1;
             }
         }
         if (tid == 0) {
@@ -780,10 +898,49 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         __syncthreads();
     }
 
-    // ---- finalise: one warp moves the row's cursor to the chosen child
+    // ---- finalise: stage 2 of the sampling, then one warp moves the row's cursor to the child
     if (warp == 0) {
-        int32_t tok = red_i[0][0], child = red_i[1][0];
-        if (tok < 0) { tok = __ldg(p.node_tok + cb); child = cb; }     // no finite score: lowest id
+        const int32_t key = red_i[0][0];
+        int32_t tok = -1, child = -1;
+        if (key < 0) {
+            tok = __ldg(p.node_tok + cb); child = cb;                 // no group with a finite score: lowest id
+        } else if (!dense) {
+            tok = key; child = red_i[1][0];                           // drawn in the gather loop already
+        } else {
+            // stage 2 for a dense row: the winning group's allowed tokens (ascending) and their
+            // weights against the group's largest logit
+            const int32_t Gw = key;
+            const uint32_t bits = mask_byte(gmask, uint32_t(Gw));
+            float xs[GROUP];
+            float xm = -CUDART_INF_F;
+#pragma unroll
+            for (int j = 0; j < GROUP; ++j) {
+                const bool on = ((bits >> j) & 1u) && Gw * GROUP + j < p.V;
+                xs[j] = on ? E::load(g.rowp, Gw * GROUP + j) : -CUDART_INF_F;
+                xm = fmaxf(xm, xs[j]);
+            }
+            const float ref = xm * p.c2;
+            float cum[GROUP];
+            float total = 0.f;
+            int last = -1, first = -1;
+#pragma unroll
+            for (int j = 0; j < GROUP; ++j) {
+                const bool on = (bits >> j) & 1u;
+                if (on) { total += exp2f(fmaf(xs[j], p.c2, -ref)); last = j; if (first < 0) first = j; }
+                cum[j] = total;
+            }
+            int pick = first;
+            if (total > 0.f && total < CUDART_INF_F) {
+                const uint4 u4 = philox4x32_10(uint32_t(Gw), r.step, r.row, 3u, p.rk);
+                const float target = uniform_from_bits(u4.x) * total;
+                pick = last;
+#pragma unroll
+                for (int j = GROUP - 1; j >= 0; --j)
+                    if (((bits >> j) & 1u) && cum[j] > target) pick = j;
+            }
+            if (pick >= 0) tok = Gw * GROUP + pick;
+            else { tok = __ldg(p.node_tok + cb); child = cb; }
+        }
         if (child < 0) {
             child = (node == 0) ? __ldg(p.root_child + tok) : warp_find_child(p.node_tok, cb, ce, tok);
         }
@@ -828,13 +985,13 @@ __global__ void k_state_init(int64_t n, int32_t N, int32_t* node, int32_t* lo, i
     node[i] = 0; lo[i] = 0; hi[i] = N; depth[i] = 0; logw[i] = 0.f; done[i] = 0;
 }
 
-__global__ void k_sampling_uniforms(PhiloxRoundKeys rk, uint32_t step, uint32_t row, int32_t v0, int32_t n,
+__global__ void k_sampling_uniforms(PhiloxRoundKeys rk, uint32_t step, uint32_t row, int32_t g0, int32_t n,
                                     float* out) {
     int i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i >= n) return;
-    uint32_t v = uint32_t(v0 + i);
-    uint4 r = philox4x32_10(v >> 2, step, row, 0u, rk);
-    out[i] = uniform_from_bits(pick_word(r, v & 3));
+    const uint32_t G = uint32_t(g0 + i);
+    const uint4 r = philox4x32_10(group_slot(G), step, row, 0u, rk);
+    out[i] = uniform_from_bits(pick_word(r, group_word(G)));
 }
 
 template <int DT, bool RING>
@@ -893,12 +1050,12 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     return ring ? launch_step<DISC_BF16, true>(p, n, smem, st) : launch_step<DISC_BF16, false>(p, n, smem, st);
 }
 
-int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t v0, int32_t n, float* out,
+int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t g0, int32_t n, float* out,
                            void* stream) {
-    if (n < 0 || v0 < 0 || (n > 0 && !out)) return DISC_ERR_ARG;
+    if (n < 0 || g0 < 0 || (n > 0 && !out)) return DISC_ERR_ARG;
     if (n == 0) return DISC_OK;
     k_sampling_uniforms<<<(n + 255) / 256, 256, 0, static_cast<cudaStream_t>(stream)>>>(philox_round_keys(seed),
-                                                                                       step, row, v0, n, out);
+                                                                                       step, row, g0, n, out);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }

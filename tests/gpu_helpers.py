@@ -25,6 +25,25 @@ def close(a, b, tol=TOL):
     return ok | same_special
 
 
+def assert_near_ties(gpu_tokens, o, sel):
+    """The rows in `sel` got a token that differs from the oracle's.  That is accepted only when
+    the oracle itself sees a near-tie (and counted): a different token group needs the oracle's
+    score of that group within TOL of the winning score; a different token of the same group needs
+    the in-group threshold within TOL (relative to the group's mass) of an interval boundary and a
+    neighbouring pick.  Rows with NaN/+Inf logits promise no particular token.  Returns the count."""
+    idx = np.nonzero(sel)[0]
+    n = 0
+    for t, i in zip(gpu_tokens, idx):
+        if o["status"][i] & 4:
+            continue
+        if (int(t) >> 3) != (int(o["token"][i]) >> 3):
+            assert o["best"][i] - o["alt"][i] < TOL, ("group", i, int(t), int(o["token"][i]), o["best"][i], o["alt"][i])
+        else:
+            assert o["ingroup_gap"][i] < TOL, ("in-group", i, int(t), int(o["token"][i]), o["ingroup_gap"][i])
+        n += 1
+    return n
+
+
 class LockStep:
     """Runs a decode on the GPU and checks every step against the oracle from the same state."""
 
@@ -64,9 +83,7 @@ class LockStep:
         same = g_tok[rows] == o["token"]
         tie = live & ~same
         if tie.any():
-            # allowed only when the oracle scores the GPU's token within TOL of its best
-            assert np.all(o["best"][tie] - o["alt"][tie] < TOL), (o["best"][tie], o["alt"][tie])
-            self.near_ties += int(tie.sum())
+            self.near_ties += assert_near_ties(g_tok[rows][tie], o, tie)
         self.checked += int(live.sum())
         exp_logw = before["logw"][rows].astype(np.float64) + o["log_mass"]
         ok = close(after["logw"][rows][live], exp_logw[live])

@@ -11,7 +11,7 @@ import torch
 
 import oracle
 import paper_2504_09135_b200 as disc
-from gpu_helpers import TOL, LockStep, close, logits_to_host
+from gpu_helpers import TOL, LockStep, assert_near_ties, close, logits_to_host
 from helpers import csr, rows_of
 from workloads import CONFIGS, make_contexts, make_lm_weights, make_prefixes, make_set, scaled
 from workloads.standin_lm import StandInLM
@@ -63,9 +63,9 @@ def test_duplicates_collapse():
 
 def test_sampling_uniforms_bit_exact():
     seed = 0xDEADBEEF12345678
-    for step, row, v0, n in [(0, 0, 0, 257), (5, 4095, 128_000, 256), (15, 123456, 7, 33)]:
-        g = disc.disc_sampling_uniforms(seed, step, row, v0, n).cpu().numpy()
-        o = np.array([oracle.gumbel_uniform(seed, step, row, v0 + i) for i in range(n)])
+    for step, row, g0, n in [(0, 0, 0, 1300), (5, 4095, 15_900, 256), (15, 123456, 7, 33)]:
+        g = disc.disc_sampling_uniforms(seed, step, row, g0, n).cpu().numpy()
+        o = np.array([oracle.group_uniform(seed, step, row, g0 + i) for i in range(n)])
         assert np.array_equal(g.astype(np.float64), o)
 
 
@@ -206,7 +206,7 @@ def test_step_layouts_and_degenerate_rows(dtype, V):
             assert np.array_equal(out.mask.cpu().numpy().view(np.uint32), m)
         assert np.array_equal(out.status.cpu().numpy(), o["status"])
         same = out.token.cpu().numpy() == o["token"]
-        assert np.all(o["best"][~same] - o["alt"][~same] < TOL)
+        assert assert_near_ties(out.token.cpu().numpy()[~same], o, ~same) <= 1
         assert close(st.logw.cpu().numpy(), o["log_mass"]).all(), (st.logw.cpu().numpy(), o["log_mass"])
         assert close(out.logq.cpu().numpy()[same], o["logq"][same]).all()
         assert close(out.logp.cpu().numpy()[same], o["logp"][same]).all()
