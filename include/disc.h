@@ -133,7 +133,11 @@ int disc_state_init(const disc_set_t* s, int64_t n, int32_t* node, int32_t* lo, 
  *   node_out    device, int32[n] (nullable): index node of the prefix (the cursor disc_step uses)
  *   status_out  device, uint8[n]: 0, or DISC_ROW_DEAD when the prefix is a prefix of no member
  *               (then the mask is zero and lo = hi = node = -1)
- * A complete member has an empty mask and a range of one row. */
+ * A complete member has an empty mask and a range of one row.
+ * With mask_out given, the call keeps a row counter in the set handle: two such calls on the
+ * same handle must not run on the device at the same time (calls issued to one stream never do;
+ * calls on different streams need an event between them, or a handle each).  n must be below
+ * 2^31 - 65536 (DISC_ERR_UNSUPPORTED otherwise). */
 int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
               const int32_t* prefix_len, int64_t n, uint32_t* mask_out, int32_t* lo_out,
               int32_t* hi_out, int32_t* node_out, uint8_t* status_out, void* stream);

@@ -416,8 +416,15 @@ int build_impl(const int32_t* tokens, const int64_t* row_offsets, int64_t n, int
         }
     }
 
+    // scratch of disc_mask: a row counter its writer kernel draws work from (see disc_mask.cu)
+    DevBuf work_counter;
+    DISC_CUDA(work_counter.alloc(256));
+    DISC_CUDA(cudaMemsetAsync(work_counter.p, 0, 256, st));
+    DISC_CUDA(cudaStreamSynchronize(st));
+    S->work_counter = static_cast<unsigned int*>(work_counter.take());
+
     S->device_bytes = int64_t(tok.bytes + row_off.bytes + node_tok.bytes + node_lo.bytes + child_begin.bytes +
-                              root_mask.bytes + root_child.bytes + heavy_nodes.bytes + heavy_masks.bytes);
+                              root_mask.bytes + root_child.bytes + heavy_nodes.bytes + heavy_masks.bytes + 256);
     S->heavy_nodes = static_cast<int32_t*>(heavy_nodes.take());
     S->heavy_masks = static_cast<uint32_t*>(heavy_masks.take());
     S->tok = static_cast<int32_t*>(tok.take());
@@ -466,6 +473,7 @@ void disc_free_set(disc_set_t* s) {
     cudaFree(s->root_child);
     cudaFree(s->heavy_nodes);
     cudaFree(s->heavy_masks);
+    cudaFree(s->work_counter);
     delete s;
 }
 

@@ -30,7 +30,10 @@ struct disc_set {
     // prebuilt masks of the nodes with more than DISC_HEAVY_MIN children ("heavy" nodes)
     int32_t n_heavy = 0;
     int32_t* heavy_nodes = nullptr;  // [n_heavy] ascending node ids
-    uint32_t* heavy_masks = nullptr; // [n_heavy][W]
+    uint32_t* heavy_masks = nullptr; // [n_heavy][Wp]
+    // scratch of disc_mask: rows handed out so far by its writer kernel (reset by its search
+    // kernel).  Calls of disc_mask on one handle must therefore not overlap on the GPU.
+    unsigned int* work_counter = nullptr;
     int64_t level_off[DISC_MAX_DEPTH + 2] = {0};  // node id where level d starts (level_off[0] = 1)
     int64_t device_bytes = 0;
     double build_seconds = 0.0;
