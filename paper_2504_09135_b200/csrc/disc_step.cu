@@ -233,6 +233,7 @@ struct Acc {
     float2 sa = {0.f, 0.f}, sb = {0.f, 0.f};      // four partial sums over all logits
     float2 ok2 = {0.f, 0.f};                      // two partial sums over the allowed logits
     bool touched = false;
+    bool improved = false;   // bound_best rose since the warp last shared its bounds
     // sampling
     Best best{-__builtin_huge_valf(), -1, -1};
     float bound_best = -__builtin_huge_valf();   // best score known to this warp (>= best.score)
@@ -264,7 +265,7 @@ __device__ __forceinline__ void exact_group(Acc& a, float t, uint32_t word, int3
     // lowest valid token at the end.
     const float score = group_score(a.cbase + log2f(t), word);
     if (score > a.best.score) { a.best.score = score; a.best.key = G; a.best.child = -1; }
-    if (score > a.bound_best) { a.bound_best = score; update_bound(a); }
+    if (score > a.bound_best) { a.bound_best = score; a.improved = true; update_bound(a); }
 }
 
 // skip test + exact evaluation of one group
@@ -537,13 +538,22 @@ __device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, 
                 if (!(tmax * a.cbound < TWO_M24)) {
                     const uint32_t G0 = uint32_t(c * GPC + tid);
                     const uint4 w4 = philox4x32_10(group_slot(G0), r.step, r.row, 0u, rk);
+                    // One test for all groups of the chunk first: the largest of the four words
+                    // gives the smallest w, the largest group mass the largest right-hand side.
+                    const uint32_t wmax = max(max(w4.x, w4.y), max(w4.z, w4.w));
+                    if (!(complement_uniform(wmax) >= tmax * a.cbound)) {
 #pragma unroll
-                    for (int j = 0; j < GPT; ++j) {
-                        const uint32_t G = G0 + uint32_t(j * STEP_THREADS);
-                        if (bits[j]) sample_group(a, tg[j], pick_word(w4, group_word(G)), int32_t(G));
+                        for (int j = 0; j < GPT; ++j) {
+                            const uint32_t G = G0 + uint32_t(j * STEP_THREADS);
+                            sample_group(a, tg[j], pick_word(w4, group_word(G)), int32_t(G));
+                        }
                     }
                 }
-                share_bound(a);
+                // a better score found by any lane tightens the whole warp's bound
+                if (__any_sync(0xffffffffu, a.improved)) {
+                    share_bound(a);
+                    a.improved = false;
+                }
             }
         };
         if (c < n_full) body(std::true_type{}); else body(std::false_type{});
