@@ -57,6 +57,18 @@ class DiscDecoder:
             self.step(logits, t, seed=seed, inv_temperature=inv_temperature)
         return self.finish(seed=seed)
 
+    def capture(self, logits_per_step, *, seed=0, inv_temperature=1.0) -> "torch.cuda.CUDAGraph":
+        """The same decode recorded once as a CUDA graph (state init, every step, resampling);
+        `graph.replay()` then enqueues the whole decode with one call.  The logits tensors, the
+        seed and this decoder's buffers are baked in: refill the logits in place between replays.
+        Results land in `self.res`, `self.seq` and `self.state` as usual."""
+        self.replay(logits_per_step, seed=seed, inv_temperature=inv_temperature)   # first-call set-up outside the capture
+        torch.cuda.synchronize(self.device)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            self.replay(logits_per_step, seed=seed, inv_temperature=inv_temperature)
+        return graph
+
     def replay_from_host(self, host_logits_per_step, staging: torch.Tensor, *, seed=0, inv_temperature=1.0):
         """Same decode with every step's logits copied from (pinned) host memory first, and the
         result read back to the host at the end."""
