@@ -46,14 +46,37 @@ struct MaskParams {
     unsigned int* work_counter;   // rows handed out so far by the writer kernel
 };
 
-// index of the child with token t among the sorted children [cb, ce), or -1 (one thread)
+// index of the child with token t among the sorted children [cb, ce), or -1 (one thread).
+// A walk is a chain of dependent loads, so each round probes eight evenly spaced keys at once
+// (independent loads, one latency) and keeps the ninth of the range that can still hold t: a
+// node with 80,000 children takes 5 rounds instead of the 17 of a binary search.
 __device__ __forceinline__ int32_t find_child(const int32_t* __restrict__ node_tok, int32_t cb, int32_t ce, int32_t t) {
-    int32_t a = cb, b = ce;
-    while (a < b) {
-        const int32_t m = (a + b) >> 1;
-        if (__ldg(node_tok + m) < t) a = m + 1; else b = m;
+    constexpr int P = 8;
+    int32_t a = cb, b = ce;                 // the first key >= t, if any, is in [a, b]
+    while (b - a > P) {
+        const int32_t s = (b - a + P) / (P + 1);          // >= 1; probe j sits at a + (j+1)*s - 1
+        int32_t key[P];
+#pragma unroll
+        for (int j = 0; j < P; ++j) {
+            const int32_t q = a + (j + 1) * s - 1;
+            key[j] = q < b ? __ldg(node_tok + q) : 0x7fffffff;
+        }
+        int cnt = 0;                        // probes with key < t form a prefix of the probes
+#pragma unroll
+        for (int j = 0; j < P; ++j) cnt += key[j] < t ? 1 : 0;
+        const int32_t na = a + cnt * s;                     // one past the last probe below t
+        const int32_t nb = cnt < P ? min(b, a + (cnt + 1) * s - 1) : b;   // the first probe not below t, if any
+        a = na;
+        b = nb;
     }
-    return (a < ce && __ldg(node_tok + a) == t) ? a : -1;
+    int32_t key[P + 1];
+#pragma unroll
+    for (int j = 0; j <= P; ++j) key[j] = (a + j < ce) ? __ldg(node_tok + a + j) : 0x7fffffff;
+    int32_t hit = -1;
+#pragma unroll
+    for (int j = P; j >= 0; --j)
+        if (a + j <= b && key[j] == t) hit = a + j;
+    return hit;
 }
 
 __device__ __forceinline__ void st_stream16(uint4* p, const uint4& v) {
@@ -314,14 +337,17 @@ extern "C" int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t pre
     int dev = 0, sms = 0;
     DISC_CUDA(cudaGetDevice(&dev));
     DISC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
-    const int64_t want = (n + MASK_WARPS * WRITE_BATCH - 1) / (MASK_WARPS * WRITE_BATCH);
-    const int64_t resident = int64_t(sms) * (2048 / MASK_THREADS);
-    const unsigned grid = unsigned(want < resident ? want : resident);
     const bool vec = (reinterpret_cast<uintptr_t>(mask_out) % 16 == 0) && (s->W % 4 == 0);
-    if (vec && head) disc_mask_write_kernel<true, true><<<grid, MASK_THREADS, 0, st>>>(p);
-    else if (vec) disc_mask_write_kernel<true, false><<<grid, MASK_THREADS, 0, st>>>(p);
-    else if (head) disc_mask_write_kernel<false, true><<<grid, MASK_THREADS, 0, st>>>(p);
-    else disc_mask_write_kernel<false, false><<<grid, MASK_THREADS, 0, st>>>(p);
+    void (*kern)(const MaskParams) = vec ? (head ? disc_mask_write_kernel<true, true> : disc_mask_write_kernel<true, false>)
+                                         : (head ? disc_mask_write_kernel<false, true> : disc_mask_write_kernel<false, false>);
+    // one wave of blocks: they share the rows through the counter
+    int per_sm = 0;
+    DISC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MASK_THREADS, 0));
+    if (per_sm < 1) per_sm = 1;
+    const int64_t want = (n + MASK_WARPS * WRITE_BATCH - 1) / (MASK_WARPS * WRITE_BATCH);
+    const int64_t resident = int64_t(sms) * per_sm;
+    const unsigned grid = unsigned(want < resident ? want : resident);
+    kern<<<grid, MASK_THREADS, 0, st>>>(p);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }
