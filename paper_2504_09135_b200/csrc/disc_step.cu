@@ -4,10 +4,12 @@
 // prefix.
 //
 // One thread block per row.
-//   * Streaming.  The row's logits are pulled into a shared-memory ring by bulk asynchronous
-//     copies (cp.async.bulk + mbarrier, one elected thread issues them), so several chunks are in
-//     flight per block whatever the register budget.  The first chunks are issued before the
-//     block reads the prefix index.  Rows that are not 16-byte aligned take a scalar-load path.
+//   * Streaming.  Thread t of the block reads the 16-byte vectors t, t+256, t+512, t+768 of every
+//     16 KB chunk of the row with plain read-only vector loads: four independent loads per thread
+//     and four blocks per SM keep some 64 KB per SM in flight, which is what HBM needs.  (A
+//     shared-memory ring filled by bulk asynchronous copies was measured slower than this on
+//     the same data, and needed waits that this version does not have.)  Rows that are not
+//     16-byte aligned take a scalar-load path.
 //   * Sums.  Each thread accumulates sum 2^(x*c - ref) against its own reference (the maximum of
 //     the first logits it sees), c = log2(e)/T.  Per pair of logits: two unpack operations, one
 //     packed fp32x2 FMA, two ex2 and one packed add.  Partial sums are kept as (m, s) pairs meaning
@@ -15,8 +17,8 @@
 //     value is added, so a common offset of the logits does not cost accuracy.
 //   * Valid set.  The prefix index gives the row's children as a contiguous list.  Rows with at
 //     most DISC_HEAVY_MIN children gather their few logits directly ("gather path").  Rows with
-//     more have a prebuilt bitmask row in global memory; its slice travels into the ring stage next
-//     to the logits it covers ("dense path").
+//     more have a prebuilt bitmask row in global memory (a few MB in total, L2 resident), read
+//     one byte per group of 8 tokens next to the logits it covers ("dense path").
 //   * Sampling (exact draw from P.mask/|P.mask|_1, Algorithm 1 line 7) in two stages.  Stage 1 is
 //     Gumbel-max over groups of 8 consecutive token ids: score_G = log(allowed mass of G) + g_G,
 //     g_G = -log(-log u_G), u_G from Philox4x32-10 keyed by (group, step, row); the best group
@@ -25,8 +27,8 @@
 //     win: with w = 1 - u, g > t implies w < e^-t, so a group whose w is at least
 //     mass_G / e^best (times a safety factor) is skipped without taking a logarithm; mass_G is
 //     the already accumulated sum of 2^(x*c - ref) times a per-thread constant.  `best` is the
-//     best score any lane of the warp has seen (shared once per chunk).  The four groups a thread
-//     owns in one chunk share one Philox counter.
+//     best score any lane of the warp has seen (shared when a lane improves it).  The four
+//     groups a thread owns in one chunk share one Philox counter.
 //   * A row whose fast sums are not finite, or whose valid mass is so small that terms may have
 //     underflowed against a thread's reference, is redone by a plain two-pass routine with exact
 //     scores ("careful path").
@@ -37,28 +39,27 @@
 
 #include "disc_internal.cuh"
 
-#ifndef DISC_STAGES
-#define DISC_STAGES 3
-#endif
+// 128 threads per row and 10 blocks per SM (48 registers per thread) measured best on B200: small
+// blocks keep the share of time a block spends outside its streaming loop low, ten of them keep
+// 1280 threads x 64 bytes in flight per SM.
 #ifndef DISC_MIN_BLOCKS
-#define DISC_MIN_BLOCKS 4
+#define DISC_MIN_BLOCKS 10
 #endif
 
 namespace {
 
 using namespace disc;
 
-constexpr int STEP_THREADS = 256;
+#ifndef DISC_STEP_THREADS
+#define DISC_STEP_THREADS 128
+#endif
+constexpr int STEP_THREADS = DISC_STEP_THREADS;
 constexpr int STEP_WARPS = STEP_THREADS / 32;
-constexpr int VPT = 4;                                   // 16-byte vectors per thread and stage
-constexpr int CHUNK_VECS = VPT * STEP_THREADS;
-constexpr int CHUNK_BYTES = CHUNK_VECS * 16;             // logits of one ring stage: 16 KB
-constexpr int MASK_SLICE_MAX = CHUNK_VECS;               // mask bytes of one stage (bf16: 8 tokens per vector)
-constexpr int STAGE_BYTES = CHUNK_BYTES + MASK_SLICE_MAX;
-constexpr int STAGES = DISC_STAGES;
-constexpr int RING_BYTES = STAGE_BYTES * STAGES;
+constexpr int VPT = 4;                                   // 16-byte vectors in flight per thread
+constexpr int SLOTS = 256;                               // a chunk is SLOTS x VPT vectors = 16 KB of the row;
+constexpr int CHUNK_VECS = VPT * SLOTS;                  // slot s owns vectors s, s+256, s+512, s+768 of it
+static_assert(SLOTS % STEP_THREADS == 0 && STEP_THREADS % 32 == 0, "a block covers a chunk in whole passes");
 constexpr int GROUP = 8;                                 // tokens per sampling group
-constexpr uint64_t WAIT_LIMIT_NS = 250ull * 1000 * 1000;  // an mbarrier wait gives up after 0.25 s
 constexpr float LOG2E_F = 1.4426950408889634f;
 constexpr float LN2_F = 0.6931471805599453f;
 constexpr float SAFETY = 1.0009765625f;                 // 1 + 2^-10 on the skip bound
@@ -131,50 +132,6 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
-// ---- mbarrier / bulk-copy wrappers -------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return uint32_t(__cvta_generic_to_shared(p)); }
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ uint64_t global_ns() {
-    uint64_t t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait: gives up (returns false) after WAIT_LIMIT_NS without the phase completing.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity) {
-    const uint64_t t0 = global_ns();
-    while (!mbar_try_wait(bar, parity)) {
-        if (global_ns() - t0 > WAIT_LIMIT_NS) return false;
-    }
-    return true;
-}
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    return mbar_try_wait(bar, parity) ? true : mbar_wait_slow(bar, parity);
-}
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void* src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-
 // ---- element types ------------------------------------------------------------------------------
 template <int DT>
 struct Elem;
@@ -206,7 +163,7 @@ struct Elem<DISC_BF16> {
 };
 
 // ---- sampling helpers ---------------------------------------------------------------------------
-// Philox counter word 0 and output word of group G.  The four groups a thread owns in one ring
+// Philox counter word 0 and output word of group G.  The four groups a thread owns in one
 // chunk (256 apart) share a counter.
 __device__ __forceinline__ uint32_t group_slot(uint32_t G) { return ((G >> 10) << 8) | (G & 255u); }
 __device__ __forceinline__ uint32_t group_word(uint32_t G) { return (G >> 8) & 3u; }
@@ -410,98 +367,58 @@ __device__ int32_t warp_find_child(const int32_t* __restrict__ node_tok, int32_t
 }
 
 // ---- streaming loops ---------------------------------------------------------------------------
-struct RingGeom {
-    const char* rowp;        // the row's logits
-    const char* gmask;       // the row's prebuilt mask (dense rows), else nullptr
-    uint32_t vec_bytes;      // bytes of the row that go through the ring (whole groups of 8 tokens)
-    uint32_t mask_bytes;     // bytes of the mask row that may be read (a multiple of 16)
-    uint32_t slice;          // mask bytes per full chunk
-    uint32_t ring_s, full_s; // shared-memory addresses of the ring and of the full barriers
-};
-
-// copy chunk c of the row (and, for dense rows, the mask slice covering it) into ring stage s and
-// arm the stage's full barrier (one thread)
-__device__ __forceinline__ void ring_issue(const RingGeom& g, int c, int s, bool with_mask) {
-    const uint32_t off = uint32_t(c) * CHUNK_BYTES;
-    const uint32_t bytes = min(uint32_t(CHUNK_BYTES), g.vec_bytes - off);
-    const uint32_t bar = g.full_s + 8u * s;
-    const uint32_t dst = g.ring_s + uint32_t(s) * STAGE_BYTES;
-    uint32_t mbytes = 0, moff = 0;
-    if (with_mask) {
-        moff = uint32_t(c) * g.slice;
-        mbytes = moff < g.mask_bytes ? min(g.slice, g.mask_bytes - moff) : 0u;
-    }
-    mbar_expect_tx(bar, bytes + mbytes);
-    bulk_g2s(dst, g.rowp + off, bytes, bar);
-    if (mbytes) bulk_g2s(dst + CHUNK_BYTES, g.gmask + moff, mbytes, bar);
+// 16-byte read-only load of streamed data (not worth keeping in L1)
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
 }
 
-// Bulk-copy ring.  Chunk c of the row lives in stage c % STAGES.  The logits of the first STAGES
-// chunks are issued by the kernel's prologue before the prefix index is read, and (for dense rows)
-// their mask slices right after it, on a barrier of their own (mask0).  Then thread 0 keeps
-// STAGES-1 chunks in flight: after every warp has copied chunk c-1 out of its stage (empty
-// barrier), that stage is refilled with chunk c-1+STAGES.  Returns false if a wait gave up.
-//
-// Work split inside a chunk.  Sparse rows: thread t takes vectors t, t+256, t+512, t+768.  Dense
-// rows work on groups of 8 tokens: bf16 - the same four vectors (one group each); f32 - groups t
-// and t+256 of the chunk's 512 (two adjacent vectors each).  Either way the groups of one thread
-// in one chunk are 256 apart and share a Philox counter.
+// The first n_groups whole groups of the row, read with 16-byte loads.
+// Work split inside a chunk of CHUNK_VECS vectors: a block passes over the chunk's 256 slots,
+// STEP_THREADS at a time.  Sparse rows: slot s takes vectors s, s+256, s+512, s+768.  Dense rows
+// work on groups of 8 tokens: bf16 - the same four vectors (one group each); f32 - groups s and
+// s+256 of the chunk's 512 (two adjacent vectors each).  Either way the groups of one slot are
+// 256 apart and share a Philox counter.
 template <int DT, bool DENSE>
-__device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const RingGeom& g, int V,
-                            const unsigned char* ring, uint32_t empty_s, uint32_t mask0_s) {
+__device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp,
+                                           const uint32_t* gmask, int n_groups) {
     using E = Elem<DT>;
     constexpr int EPV = E::EPV;
     constexpr int NP = EPV / 2;
     constexpr int VPG = GROUP / EPV;                          // vectors per group: 1 (bf16) or 2 (f32)
     constexpr int GPT = VPT / VPG;                            // groups per thread and chunk
-    constexpr int GPC = GPT * STEP_THREADS;                   // groups per chunk
-    const int tid = threadIdx.x, lane = tid & 31;
-    const int nvec = int(g.vec_bytes / 16u);
-    const int ngroups = nvec / VPG;
-    const int n_chunks = int((g.vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
-    const int n_full = int(g.vec_bytes / CHUNK_BYTES);
-    bool ok = true;
+    constexpr int GPC = GPT * SLOTS;                          // groups per chunk
+    const uint4* row4 = reinterpret_cast<const uint4*>(rowp);
+    const unsigned char* gbytes = reinterpret_cast<const unsigned char*>(gmask);
+    const int nvec = n_groups * VPG;
+    const int n_chunks = (nvec + CHUNK_VECS - 1) / CHUNK_VECS;
+    const int n_full = nvec / CHUNK_VECS;
 
-    // the mask slices of the first STAGES chunks were copied separately (see the kernel's prologue)
-    if constexpr (DENSE) {
-        if (!__all_sync(0xffffffffu, mbar_wait(mask0_s, 0u))) return false;
-    }
-
-    int s = 0, sp = STAGES - 1;          // stage of chunk c and of chunk c-1
-    uint32_t ph = 0, php = 1;            // their phase parities (php is only used from c = 1 on)
     for (int c = 0; c < n_chunks; ++c) {
-        // the give-up decision is taken per warp, so that all lanes leave the loop together
-        if (!__all_sync(0xffffffffu, mbar_wait(g.full_s + 8u * s, ph))) { ok = false; break; }
-        const unsigned char* stage_b = ring + s * STAGE_BYTES;
-        const uint4* stage = reinterpret_cast<const uint4*>(stage_b);
-
-        auto body = [&](auto full_tag) {
+        auto body = [&](auto full_tag, int slot) {
             constexpr bool FULL = decltype(full_tag)::value;
             uint4 raw[VPT];
             uint32_t bits[GPT];
             bool have[VPT];
             // vector index inside the chunk of this thread's k-th vector
-            auto vidx = [&](int k) { return DENSE ? ((k / VPG) * STEP_THREADS + tid) * VPG + (k % VPG)
-                                                  : k * STEP_THREADS + tid; };
+            auto vidx = [&](int k) { return DENSE ? ((k / VPG) * SLOTS + slot) * VPG + (k % VPG)
+                                                  : k * SLOTS + slot; };
 #pragma unroll
             for (int k = 0; k < VPT; ++k) {
                 have[k] = FULL || (c * CHUNK_VECS + vidx(k) < nvec);
-                if (have[k]) raw[k] = stage[vidx(k)];
+                if (have[k]) raw[k] = ld_stream16(row4 + c * CHUNK_VECS + vidx(k));
             }
             if constexpr (DENSE) {
 #pragma unroll
                 for (int j = 0; j < GPT; ++j) {
-                    const int gi = j * STEP_THREADS + tid;           // group index inside the chunk
-                    bits[j] = (FULL || c * GPC + gi < ngroups) ? uint32_t(stage_b[CHUNK_BYTES + gi]) : 0u;
+                    const int G = c * GPC + j * SLOTS + slot;
+                    bits[j] = (FULL || G < n_groups) ? uint32_t(__ldg(gbytes + G)) : 0u;
                 }
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(empty_s + 8u * s);
-            if (tid == 0 && c >= 1 && c - 1 + STAGES < n_chunks) {
-                if (!mbar_wait(empty_s + 8u * sp, php)) ok = false;
-                else ring_issue(g, c - 1 + STAGES, sp, DENSE);
-            }
-            if (c == 0 && have[0]) {
+            if (!a.touched && have[0]) {
                 float2 x[NP];
                 E::unpack(raw[0], x);
                 float mx = fmaxf(x[0].x, x[0].y);
@@ -536,7 +453,7 @@ __device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, 
 #pragma unroll
                 for (int j = 1; j < GPT; ++j) tmax = fmaxf(tmax, tg[j]);
                 if (!(tmax * a.cbound < TWO_M24)) {
-                    const uint32_t G0 = uint32_t(c * GPC + tid);
+                    const uint32_t G0 = uint32_t(c * GPC + slot);
                     const uint4 w4 = philox4x32_10(group_slot(G0), r.step, r.row, 0u, rk);
                     // One test for all groups of the chunk first: the largest of the four words
                     // gives the smallest w, the largest group mass the largest right-hand side.
@@ -544,7 +461,7 @@ __device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, 
                     if (!(complement_uniform(wmax) >= tmax * a.cbound)) {
 #pragma unroll
                         for (int j = 0; j < GPT; ++j) {
-                            const uint32_t G = G0 + uint32_t(j * STEP_THREADS);
+                            const uint32_t G = G0 + uint32_t(j * SLOTS);
                             sample_group(a, tg[j], pick_word(w4, group_word(G)), int32_t(G));
                         }
                     }
@@ -556,16 +473,14 @@ __device__ bool stream_ring(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, 
                 }
             }
         };
-        if (c < n_full) body(std::true_type{}); else body(std::false_type{});
-
-        sp = s; php = ph;
-        if (++s == STAGES) { s = 0; ph ^= 1u; }
+        for (int slot = threadIdx.x; slot < SLOTS; slot += STEP_THREADS) {
+            if (c < n_full) body(std::true_type{}, slot); else body(std::false_type{}, slot);
+        }
     }
-    return ok;
 }
 
 // groups [g_begin, g_end) of the row read with scalar loads (whole row on the scalar path; the
-// ragged last group on the ring path)
+// ragged last group on the vector path)
 template <int DT, bool DENSE>
 __device__ void stream_groups_scalar(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp, int V,
                                      const uint32_t* gmask, int g_begin, int g_end) {
@@ -581,19 +496,15 @@ __device__ void stream_groups_scalar(Acc& a, const RowCtx& r, const PhiloxRoundK
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
-template <int DT, bool RING>
+template <int DT, bool VEC>
 __global__ void __launch_bounds__(STEP_THREADS, DISC_MIN_BLOCKS)
 disc_step_kernel(const __grid_constant__ StepParams p) {
     using E = Elem<DT>;
-    extern __shared__ __align__(128) unsigned char ring[];        // RING_BYTES (RING only)
-    __shared__ __align__(8) uint64_t full_bar[STAGES];
-    __shared__ __align__(8) uint64_t empty_bar[STAGES];
-    __shared__ __align__(8) uint64_t mask0_bar;
     __shared__ float red_f[6][STEP_WARPS];
     __shared__ int32_t red_i[2][STEP_WARPS];
     __shared__ float scratch[STEP_WARPS];
     __shared__ float fin[4];        // (m, s) of the full row and of the valid set
-    __shared__ int32_t s_flag, s_tmp, s_fault;
+    __shared__ int32_t s_flag, s_tmp;
 
     const int64_t row = blockIdx.x;
     const int tid = threadIdx.x;
@@ -603,29 +514,9 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_DONE; }
         return;
     }
-    // Start streaming before anything else: the first ring stages fill while the index is read.
     const int n_groups = (p.V + GROUP - 1) / GROUP;       // the last one may be ragged
-    const int n_ring_groups = RING ? p.V / GROUP : 0;     // whole groups go through the ring
-    RingGeom g;
-    g.rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
-    g.gmask = nullptr;
-    g.vec_bytes = uint32_t(n_ring_groups) * uint32_t(GROUP * E::SIZE);
-    g.mask_bytes = uint32_t(p.Wp) * 4u;
-    g.slice = uint32_t(CHUNK_VECS * E::EPV / GROUP);
-    g.ring_s = smem_u32(ring);
-    g.full_s = smem_u32(full_bar);
-    const int n_chunks = int((g.vec_bytes + CHUNK_BYTES - 1) / CHUNK_BYTES);
-    if (RING && tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(smem_u32(&full_bar[s]), 1);
-            mbar_init(smem_u32(&empty_bar[s]), STEP_WARPS);
-        }
-        mbar_init(smem_u32(&mask0_bar), 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        for (int k = 0; k < STAGES && k < n_chunks; ++k) ring_issue(g, k, k, false);
-    }
-    if (tid == 0) s_fault = 0;
+    const int n_vec_groups = VEC ? p.V / GROUP : 0;       // whole groups are read with 16-byte loads
+    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
 
     const int32_t node = p.node[row];
     int32_t cb = 0, ce = 0;
@@ -637,45 +528,25 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             bool leaf = node > 0 && int64_t(node) < p.M;
             p.status_out[row] = leaf ? DISC_ROW_DONE : DISC_ROW_DEAD;
             if (leaf) p.done[row] = 1;
-            // the copies already in flight must land before the block's shared memory is released
-            if (RING)
-                for (int k = 0; k < STAGES && k < n_chunks; ++k) mbar_wait(smem_u32(&full_bar[k]), 0u);
         }
         return;
     }
 
-    // dense rows: locate the prebuilt mask row (root, or a heavy node) and fetch the mask slices of
-    // the chunks already in flight
+    // dense rows: locate the prebuilt mask row (root, or a heavy node)
     if (tid == 0) {
         int32_t h = -2;                                   // -2: not dense
         if (node == 0) h = -1;                            // -1: the root's row
         else if (c > DISC_HEAVY_MIN) { h = heavy_index(p.heavy_nodes, p.n_heavy, node); if (h < 0) h = -2; }
         s_tmp = h;
-        if (RING && h != -2) {
-            const char* gm = reinterpret_cast<const char*>(h == -1 ? p.root_mask : p.heavy_masks + size_t(h) * p.Wp);
-            uint32_t total = 0;
-            for (int k = 0; k < STAGES && k < n_chunks; ++k) {
-                const uint32_t moff = uint32_t(k) * g.slice;
-                total += moff < g.mask_bytes ? min(g.slice, g.mask_bytes - moff) : 0u;
-            }
-            const uint32_t bar = smem_u32(&mask0_bar);
-            mbar_expect_tx(bar, total);
-            for (int k = 0; k < STAGES && k < n_chunks; ++k) {
-                const uint32_t moff = uint32_t(k) * g.slice;
-                const uint32_t mb = moff < g.mask_bytes ? min(g.slice, g.mask_bytes - moff) : 0u;
-                if (mb) bulk_g2s(g.ring_s + uint32_t(k) * STAGE_BYTES + CHUNK_BYTES, gm + moff, mb, bar);
-            }
-        }
     }
     __syncthreads();
     const int32_t hsel = s_tmp;
     const bool dense = hsel != -2;
     const uint32_t* gmask = !dense ? nullptr : (hsel == -1 ? p.root_mask : p.heavy_masks + size_t(hsel) * p.Wp);
-    g.gmask = reinterpret_cast<const char*>(gmask);
 
     RowCtx r;
     r.c2 = p.c2; r.inv_t = p.inv_t; r.step = p.step; r.row = uint32_t(p.row_base + uint32_t(row));
-    r.xref = E::load(g.rowp, 0);
+    r.xref = E::load(rowp, 0);
     if (!(fabsf(r.xref) < CUDART_INF_F)) r.xref = 0.f;
 
     Acc a;
@@ -703,7 +574,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         // nothing of this is left for the end of the block.
         for (int i = tid; i < c; i += STEP_THREADS) {
             const int32_t v = __ldg(p.node_tok + cb + i);
-            const float x = E::load(g.rowp, v);
+            const float x = E::load(rowp, v);
             ms_add(ok, x, p.c2);
             const int32_t G = v >> 3;
             const bool leader = (i == 0) || ((__ldg(p.node_tok + cb + i - 1) >> 3) != G);
@@ -715,7 +586,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
                 for (int k = 1; k < GROUP; ++k) {
                     if (n == k && i + k < c) {
                         const int32_t v2 = __ldg(p.node_tok + cb + i + k);
-                        if ((v2 >> 3) == G) { xs[k] = E::load(g.rowp, v2); n = k + 1; }
+                        if ((v2 >> 3) == G) { xs[k] = E::load(rowp, v2); n = k + 1; }
                     }
                 }
                 MS gm{-CUDART_INF_F, 0.f};
@@ -754,27 +625,16 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     }
 
     // ---- stream the row
-    bool waits_ok = true;
-    if (RING) {
-        waits_ok = dense ? stream_ring<DT, true>(a, r, p.rk, g, p.V, ring, smem_u32(empty_bar), smem_u32(&mask0_bar))
-                         : stream_ring<DT, false>(a, r, p.rk, g, p.V, ring, smem_u32(empty_bar), smem_u32(&mask0_bar));
+    if (VEC) {
+        if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups);
+        else stream_vec<DT, false>(a, r, p.rk, rowp, gmask, n_vec_groups);
     }
-    if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, g.rowp, p.V, gmask, n_ring_groups, n_groups);
-    else stream_groups_scalar<DT, false>(a, r, p.rk, g.rowp, p.V, gmask, n_ring_groups, n_groups);
-    if (!waits_ok) s_fault = 1;
+    if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
+    else stream_groups_scalar<DT, false>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
 
     MS all = a.touched ? MS{a.mref, (a.sa.x + a.sa.y) + (a.sb.x + a.sb.y)} : MS{-CUDART_INF_F, 0.f};
     if (dense) ok = a.touched ? MS{a.mref, a.ok2.x + a.ok2.y} : MS{-CUDART_INF_F, 0.f};
     Best best = a.best;
-
-    __syncthreads();
-    if (s_fault) {
-        // A bulk copy never signalled completion.  Report it and leave the row untouched; give
-        // outstanding copies a bounded time to land before the block's shared memory is released.
-        for (int i = 0; i < 2000; ++i) __nanosleep(1000);
-        if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_FAULT; }
-        return;
-    }
 
     // ---- block reduction of (all, ok, best)
 #pragma unroll
@@ -841,7 +701,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         for (int G = tid; G < n_groups; G += STEP_THREADS) {
             const uint32_t bits = dense ? mask_byte(gmask, uint32_t(G)) : 0u;
             for (int j = 0; j < GROUP && G * GROUP + j < p.V; ++j) {
-                const float x = E::load(g.rowp, G * GROUP + j);
+                const float x = E::load(rowp, G * GROUP + j);
                 const bool allowed = (bits >> j) & 1u;
                 if (x != x) { nan_all = 1; nan_ok |= allowed; }
                 else { mx_all = fmaxf(mx_all, x); if (allowed) mx_ok = fmaxf(mx_ok, x); }
@@ -849,7 +709,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         }
         if (!dense) {
             for (int i = tid; i < c; i += STEP_THREADS) {
-                const float x = E::load(g.rowp, __ldg(p.node_tok + cb + i));
+                const float x = E::load(rowp, __ldg(p.node_tok + cb + i));
                 if (x != x) nan_ok = 1; else mx_ok = fmaxf(mx_ok, x);
             }
         }
@@ -865,7 +725,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             const uint32_t bits = dense ? mask_byte(gmask, uint32_t(G)) : 0u;
             float tg = 0.f;
             for (int j = 0; j < GROUP && G * GROUP + j < p.V; ++j) {
-                const float x = E::load(g.rowp, G * GROUP + j);
+                const float x = E::load(rowp, G * GROUP + j);
                 if (fin_all) sum_all += exp2f(fmaf(x, p.c2, -r_all));
                 if (fin_ok && ((bits >> j) & 1u)) tg += exp2f(fmaf(x, p.c2, -r_ok));
             }
@@ -879,7 +739,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         }
         if (!dense && fin_ok) {
             for (int i = tid; i < c; i += STEP_THREADS)
-                sum_ok += exp2f(fmaf(E::load(g.rowp, __ldg(p.node_tok + cb + i)), p.c2, -r_ok));
+                sum_ok += exp2f(fmaf(E::load(rowp, __ldg(p.node_tok + cb + i)), p.c2, -r_ok));
         }
         sum_all = block_sum(sum_all, scratch);
         sum_ok = block_sum(sum_ok, scratch);
@@ -926,7 +786,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 #pragma unroll
             for (int j = 0; j < GROUP; ++j) {
                 const bool on = ((bits >> j) & 1u) && Gw * GROUP + j < p.V;
-                xs[j] = on ? E::load(g.rowp, Gw * GROUP + j) : -CUDART_INF_F;
+                xs[j] = on ? E::load(rowp, Gw * GROUP + j) : -CUDART_INF_F;
                 xm = fmaxf(xm, xs[j]);
             }
             const float ref = xm * p.c2;
@@ -968,7 +828,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             uint8_t st = 0;
             if (!f_all) st |= DISC_ROW_NONFINITE;
             if (!f_ok) st |= DISC_ROW_NOMASS;
-            const float xt = E::load(g.rowp, tok);
+            const float xt = E::load(rowp, tok);
             const float logq = f_ok ? (fmaf(xt, p.c2, -K.m) - lg_ok) * LN2_F : (xt * p.c2 - l2_ok) * LN2_F;
             const float logp = f_all ? (fmaf(xt, p.c2, -A.m) - lg_all) * LN2_F : (xt * p.c2 - l2_all) * LN2_F;
             const int32_t d = p.depth[row];
@@ -1004,11 +864,9 @@ __global__ void k_sampling_uniforms(PhiloxRoundKeys rk, uint32_t step, uint32_t 
     out[i] = uniform_from_bits(pick_word(r, group_word(G)));
 }
 
-template <int DT, bool RING>
-int launch_step(const StepParams& p, int64_t n, size_t smem, cudaStream_t st) {
-    DISC_CUDA(cudaFuncSetAttribute(disc_step_kernel<DT, RING>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                   int(smem)));
-    disc_step_kernel<DT, RING><<<unsigned(n), STEP_THREADS, smem, st>>>(p);
+template <int DT, bool VEC>
+int launch_step(const StepParams& p, int64_t n, cudaStream_t st) {
+    disc_step_kernel<DT, VEC><<<unsigned(n), STEP_THREADS, 0, st>>>(p);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }
@@ -1052,12 +910,11 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.M = s->M;
 
     const size_t esize = dtype == DISC_F32 ? 4 : 2;
-    // the bulk-copy ring needs 16-byte aligned rows; other layouts take the scalar path
-    const bool ring = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
-    const size_t smem = ring ? RING_BYTES : 0;
+    // 16-byte loads need 16-byte aligned rows; other layouts take the scalar path
+    const bool vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    if (dtype == DISC_F32) return ring ? launch_step<DISC_F32, true>(p, n, smem, st) : launch_step<DISC_F32, false>(p, n, smem, st);
-    return ring ? launch_step<DISC_BF16, true>(p, n, smem, st) : launch_step<DISC_BF16, false>(p, n, smem, st);
+    if (dtype == DISC_F32) return vec ? launch_step<DISC_F32, true>(p, n, st) : launch_step<DISC_F32, false>(p, n, st);
+    return vec ? launch_step<DISC_BF16, true>(p, n, st) : launch_step<DISC_BF16, false>(p, n, st);
 }
 
 int disc_sampling_uniforms(uint64_t seed, uint32_t step, uint32_t row, int32_t g0, int32_t n, float* out,
