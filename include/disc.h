@@ -66,8 +66,8 @@ extern "C" {
 #define DISC_ROW_NOMASS 2   /* allowed probability mass is zero or not finite                     */
 #define DISC_ROW_NONFINITE 4 /* NaN or +Inf among the row's logits (or NaN among the weights)     */
 #define DISC_ROW_DONE 8     /* row was already complete: nothing read, state untouched            */
-#define DISC_ROW_FAULT 16   /* an asynchronous copy inside the kernel never completed (bounded wait
-                               gave up); the row's state is untouched                             */
+#define DISC_ROW_FAULT 16   /* reserved for kernels that wait on asynchronous copies; the present ones
+                               have no waits and never set it                                     */
 
 typedef struct disc_set disc_set_t; /* opaque; owns its device memory */
 
