@@ -142,6 +142,27 @@ int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
               const int32_t* prefix_len, int64_t n, uint32_t* mask_out, int32_t* lo_out,
               int32_t* hi_out, int32_t* node_out, uint8_t* status_out, void* stream);
 
+/* disc_mask with the writer's row counter in a fixed word block inside the loaded module (a
+ * file-scope device array of 256 bytes per device) instead of device memory obtained from the
+ * allocator.  The paper has no counterpart of this entry point; it exists for callers that cannot
+ * let a library allocate device memory on their behalf: a serving process that sizes its own pool
+ * to all of the memory left at start-up has no room to give later, and an allocation made behind
+ * its back can fail or push it over its budget.  This call performs no allocation and frees
+ * nothing, on the device or through the CUDA allocator.
+ * Arguments, outputs and errors are those of disc_mask.  In addition:
+ *   - n must not exceed DISC_MASK_STATIC_MAX_ROWS; a larger n is refused with DISC_ERR_UNSUPPORTED
+ *     before anything is launched;
+ *   - the first call on a device looks up the address of the word block (with that device
+ *     current) and keeps it; make that first call outside any stream capture;
+ *   - the block is shared by every call on that device, whatever the handle or stream: two calls
+ *     must not run on the device at the same time (calls on one stream never do).  Nothing has to be
+ *     cleared between calls: the first kernel of each call resets the counter, and what an earlier
+ *     call left there is never read. */
+#define DISC_MASK_STATIC_MAX_ROWS 1073741824 /* 2^30 prefixes per call */
+int disc_mask_static(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
+                     const int32_t* prefix_len, int64_t n, uint32_t* mask_out, int32_t* lo_out,
+                     int32_t* hi_out, int32_t* node_out, uint8_t* status_out, void* stream);
+
 /* One decoding step for n candidates (Algorithm 1, lines 5-8; score closed form in Appendix A).
  *   logits   device, n rows of V values of type `dtype`, row i at element offset i*ld.  The fast
  *            path needs the base 16-byte aligned and ld*sizeof(value) a multiple of 16; other

@@ -24,7 +24,7 @@ ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "D
           -5: "DISC_ERR_OOM", -6: "DISC_ERR_CUDA", -7: "DISC_ERR_UNSUPPORTED"}
 
 EXPORTS = ["disc_build_set", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
-           "disc_mask", "disc_step", "disc_resample", "disc_accept", "disc_sampling_uniforms",
+           "disc_mask", "disc_mask_static", "disc_step", "disc_resample", "disc_accept", "disc_sampling_uniforms",
            "disc_error_string", "disc_last_cuda_error"]
 
 
@@ -63,6 +63,7 @@ def lib():
     L.disc_set_rows.argtypes = [vp, vp, vp]
     L.disc_state_init.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp]
     L.disc_mask.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp, vp, vp]
+    L.disc_mask_static.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp, vp, vp]
     L.disc_step.argtypes = [vp, vp, C.c_int, i64, i64, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
                             vp, vp, i32, vp, vp, vp, vp, vp]
     L.disc_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, i32, vp, vp, vp]
@@ -206,6 +207,33 @@ def disc_mask(s: DiscSet, prefix: torch.Tensor, prefix_len: torch.Tensor, *, wan
                          _dev(out["hi"], torch.int32, "hi"), _dev(out["node"], torch.int32, "node"),
                          _dev(out["status"], torch.uint8, "status"), _stream_ptr(stream))
     _check(rc, "disc_mask")
+    return out
+
+
+MASK_STATIC_MAX_ROWS = 1 << 30
+
+
+def disc_mask_static(s: DiscSet, prefix: torch.Tensor, prefix_len: torch.Tensor, *, want_mask=True, out=None,
+                     stream=None):
+    """disc_mask through the entry point that keeps its row counter in a fixed word block of the
+    library instead of allocated device memory (same arguments and results)."""
+    n = prefix_len.shape[0]
+    if n > MASK_STATIC_MAX_ROWS:
+        raise ValueError(f"disc_mask_static: {n} prefixes exceed the limit of {MASK_STATIC_MAX_ROWS} per call")
+    dev = prefix_len.device
+    ld = prefix.shape[1] if prefix.ndim == 2 else 0
+    if out is None:
+        out = {"mask": torch.empty((n, s.W), dtype=torch.int32, device=dev) if want_mask else None,
+               "lo": torch.empty(n, dtype=torch.int32, device=dev),
+               "hi": torch.empty(n, dtype=torch.int32, device=dev),
+               "node": torch.empty(n, dtype=torch.int32, device=dev),
+               "status": torch.empty(n, dtype=torch.uint8, device=dev)}
+    rc = lib().disc_mask_static(s.handle, _dev(prefix, torch.int32, "prefix") if ld > 0 else 0, ld,
+                                _dev(prefix_len, torch.int32, "prefix_len"), n,
+                                _dev(out["mask"], torch.int32, "mask"), _dev(out["lo"], torch.int32, "lo"),
+                                _dev(out["hi"], torch.int32, "hi"), _dev(out["node"], torch.int32, "node"),
+                                _dev(out["status"], torch.uint8, "status"), _stream_ptr(stream))
+    _check(rc, "disc_mask_static")
     return out
 
 

@@ -19,6 +19,8 @@
 // The counter lives in the set handle: two disc_mask calls on the same handle must not run at the
 // same time on the device (calls on one stream never do).
 
+#include <mutex>
+
 #include "disc_internal.cuh"
 
 namespace {
@@ -325,6 +327,79 @@ extern "C" int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t pre
     p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
     p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.N = int32_t(s->N);
     p.work_counter = s->work_counter;
+
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const bool head = s->W >= HEAD_WORDS;
+    const unsigned sgrid = unsigned((n + MASK_THREADS - 1) / MASK_THREADS);
+    if (head) disc_mask_search_kernel<true><<<sgrid, MASK_THREADS, 0, st>>>(p);
+    else disc_mask_search_kernel<false><<<sgrid, MASK_THREADS, 0, st>>>(p);
+    DISC_CUDA(cudaGetLastError());
+    if (!mask_out) return DISC_OK;
+
+    int dev = 0, sms = 0;
+    DISC_CUDA(cudaGetDevice(&dev));
+    DISC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const bool vec = (reinterpret_cast<uintptr_t>(mask_out) % 16 == 0) && (s->W % 4 == 0);
+    void (*kern)(const MaskParams) = vec ? (head ? disc_mask_write_kernel<true, true> : disc_mask_write_kernel<true, false>)
+                                         : (head ? disc_mask_write_kernel<false, true> : disc_mask_write_kernel<false, false>);
+    // one wave of blocks: they share the rows through the counter
+    int per_sm = 0;
+    DISC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, MASK_THREADS, 0));
+    if (per_sm < 1) per_sm = 1;
+    const int64_t want = (n + MASK_WARPS * WRITE_BATCH - 1) / (MASK_WARPS * WRITE_BATCH);
+    const int64_t resident = int64_t(sms) * per_sm;
+    const unsigned grid = unsigned(want < resident ? want : resident);
+    kern<<<grid, MASK_THREADS, 0, st>>>(p);
+    DISC_CUDA(cudaGetLastError());
+    return DISC_OK;
+}
+
+// ---- disc_mask_static: the same two kernels with the writer's row counter in a word block that is
+// part of this module's image instead of the allocation disc_build_set makes for the handle.
+namespace {
+
+// scratch of disc_mask_static, one copy per device: word 0 is the row counter, the rest is unused
+static __device__ __align__(256) unsigned int g_mask_static_scratch[64];
+
+constexpr int MAX_DEVICES = 64;
+unsigned int* g_static_ptr[MAX_DEVICES] = {nullptr};
+std::mutex g_static_mutex;
+
+// address of the scratch block on the current device; looked up once per device
+int static_counter(unsigned int** out) {
+    int dev = 0;
+    DISC_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return DISC_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (!g_static_ptr[dev]) {
+        unsigned int* ptr = nullptr;
+        DISC_CUDA(cudaGetSymbolAddress(reinterpret_cast<void**>(&ptr), g_mask_static_scratch));
+        if (!ptr) return DISC_ERR_CUDA;
+        g_static_ptr[dev] = ptr;
+    }
+    *out = g_static_ptr[dev];
+    return DISC_OK;
+}
+
+}  // namespace
+
+extern "C" int disc_mask_static(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld, const int32_t* prefix_len,
+                                int64_t n, uint32_t* mask_out, int32_t* lo_out, int32_t* hi_out,
+                                int32_t* node_out, uint8_t* status_out, void* stream) {
+    if (!s || n < 0 || prefix_ld < 0) return DISC_ERR_ARG;
+    if (n == 0) return DISC_OK;
+    if (!prefix_len || !status_out || (prefix_ld > 0 && !prefix)) return DISC_ERR_ARG;
+    if (n > DISC_MASK_STATIC_MAX_ROWS) return DISC_ERR_UNSUPPORTED;   // beyond what the static counter can hand out
+    unsigned int* counter = nullptr;
+    if (const int rc = static_counter(&counter)) return rc;
+    MaskParams p;
+    p.prefix = prefix; p.prefix_ld = prefix_ld; p.prefix_len = prefix_len; p.n = n;
+    p.mask_out = mask_out; p.lo_out = lo_out; p.hi_out = hi_out; p.node_out = node_out; p.status_out = status_out;
+    p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
+    p.root_child = s->root_child; p.root_mask = s->root_mask;
+    p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
+    p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.N = int32_t(s->N);
+    p.work_counter = counter;
 
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const bool head = s->W >= HEAD_WORDS;
