@@ -339,11 +339,12 @@ def run_ours(args):
         del host, staging
 
     # ---- mask-only stress (secondary figure): 65,536 prefixes of the same table
-    mask_stress = None
+    mask_stress, mask_sample = None, None
     if rank == 0 and w.name == "large":
         from workloads import CONFIGS, make_prefixes
         mw = CONFIGS["mask"]
         prefix, plen = make_prefixes(mw, tok, off)
+        mask_sample = (prefix[:4096], plen[:4096])
         pre_d, len_d = torch.as_tensor(prefix, device=dev), torch.as_tensor(plen, device=dev)
         out = disc.disc_mask(G, pre_d, len_d)
         torch.cuda.synchronize()
@@ -368,7 +369,7 @@ def run_ours(args):
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         seq = dec.seq.cpu().numpy()
         cpu = cpu_baseline(w, tok, off, [l[:args.cpu_sample_rows] for l in logits_steps], seq[:args.cpu_sample_rows],
-                           seed)
+                           seed, mask_sample)
 
     if rank == 0:
         line = {"metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -399,7 +400,7 @@ def run_ours(args):
 
 
 # ----------------------------------------------------------------------------- oracle on the host
-def cpu_baseline(w, tok, off, logits_rows, seq, seed):
+def cpu_baseline(w, tok, off, logits_rows, seq, seed, mask_sample=None):
     """Times oracle.step on the sampled rows over every position (teacher-forced on the GPU's own
     tokens, so each call does the work of the corresponding disc_step rows)."""
     import oracle
@@ -426,10 +427,16 @@ def cpu_baseline(w, tok, off, logits_rows, seq, seed):
     toks_all, secs_all = run(n, cores)
     n1 = max(1, n // 16)
     toks_1, secs_1 = run(n1, 1)
-    return {"value": round(toks_all / secs_all, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
-            "sample": f"first {n} of {w.R} rows, all positions ({toks_all} tokens, {secs_all:.1f} s)",
-            "value_1_thread": round(toks_1 / secs_1, 1), "sample_1_thread": f"first {n1} rows ({secs_1:.1f} s)",
-            "trie_build_s": round(build_s, 1)}
+    out = {"value": round(toks_all / secs_all, 1), "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"first {n} of {w.R} rows, all positions ({toks_all} tokens, {secs_all:.1f} s)",
+           "value_1_thread": round(toks_1 / secs_1, 1), "sample_1_thread": f"first {n1} rows ({secs_1:.1f} s)",
+           "trie_build_s": round(build_s, 1)}
+    if mask_sample is not None:      # the mask stress on one host thread (the oracle's mask walk is serial)
+        a = time.perf_counter()
+        S.mask(*mask_sample)
+        out["mask_prefixes_per_s_1_thread"] = round(mask_sample[1].shape[0] / (time.perf_counter() - a), 1)
+        out["mask_sample"] = f"first {mask_sample[1].shape[0]} of the 65,536 prefixes"
+    return out
 
 
 def run_reference(args):
