@@ -68,6 +68,8 @@ def lib():
         L.oracle_resample.restype = None
         L.oracle_accept.argtypes = [vp, i32, i32, u64, vp, vp]
         L.oracle_accept.restype = None
+        L.oracle_accept_resample.argtypes = [vp, i32, i32, u64, vp, vp, vp, vp, vp, vp]
+        L.oracle_accept_resample.restype = None
         L.oracle_decode_markov.argtypes = [vp, vp, vp, i32, i32, C.c_float, u64, i64,
                                            vp, vp, vp, vp, vp, vp, C.c_int]
         L.oracle_decode_markov.restype = C.c_int
@@ -221,6 +223,20 @@ def accept(logw, seed=0, query_ids=None):
     out = np.empty(B, np.int32)
     lib().oracle_accept(_p(logw), B, K, int(seed), _p(query_ids), _p(out))
     return out
+
+
+def accept_resample(logw, seed=0, query_ids=None):
+    """Algorithm 1, lines 11-22 on [B][2K] log-weights: the first K columns are tried in order by
+    the accept test, the last K are the fresh candidates of the K-way draw."""
+    logw = _c(logw, np.float32)
+    B, K2 = logw.shape
+    assert K2 % 2 == 0 and K2 > 0
+    query_ids = None if query_ids is None else _c(query_ids, np.int64)
+    o = {"choice": np.empty(B, np.int32), "first": np.empty(B, np.int32), "logz": np.empty(B),
+         "gap": np.empty(B), "status": np.empty(B, np.uint8)}
+    lib().oracle_accept_resample(_p(logw), B, K2 // 2, int(seed), _p(query_ids), _p(o["choice"]), _p(o["first"]),
+                                 _p(o["logz"]), _p(o["gap"]), _p(o["status"]))
+    return o
 
 
 def philox4x32_10(ctr, key):

@@ -531,6 +531,30 @@ void oracle_accept(const float* logw, int32_t B, int32_t K, uint64_t seed, const
     }
 }
 
+// Algorithm 1, lines 11-22, on 2K finished candidates per query (logw is [B][2K]): candidates
+// 0..K-1 go through the accept test in order (lines 12-20: return the first with x > eps); when
+// all K are rejected, one of the K fresh candidates K..2K-1 is drawn with probability
+// x_k / sum_j x_j (line 22).  choice[b] is the column returned, first_accepted[b] the accepted
+// candidate or -1, logz/gap/status describe the K-way draw over the fresh candidates (computed for
+// every query, used only after K rejections).
+void oracle_accept_resample(const float* logw, int32_t B, int32_t K, uint64_t seed, const int64_t* query_ids,
+                            int32_t* choice, int32_t* first_accepted, double* logz, double* gap, uint8_t* status) {
+    std::vector<double> lw(K);
+    for (int32_t b = 0; b < B; ++b) {
+        const float* w = logw + int64_t(b) * 2 * K;
+        uint32_t q = uint32_t(query_ids ? query_ids[b] : b);
+        int32_t first = -1;
+        for (int32_t k = 0; k < K && first < 0; ++k)
+            if (double(w[k]) > std::log(accept_uniform(seed, q, uint32_t(k)))) first = k;
+        for (int k = 0; k < K; ++k) lw[k] = double(w[K + k]);
+        ResampleOut o = resample_query(lw.data(), K, resample_uniform(seed, q));
+        first_accepted[b] = first;
+        choice[b] = first >= 0 ? first : K + o.idx;
+        logz[b] = o.logz; status[b] = o.status;
+        if (gap) gap[b] = o.gap;
+    }
+}
+
 // Free-running decode of B queries x K candidates under a first-order Markov language model given
 // as a table: logits of the next token after token p are Z[p*V .. +V) (fp32); the first step uses
 // the query's context token.  Runs Algorithm 1's SampleCandidate for every (query, candidate) and

@@ -171,3 +171,47 @@ def test_accept_phase_expected_draws_and_accepted_law():
         for j in range(K if k < 0 else k + 1):
             ok = np.float64(o["logw32"][b, j]) > np.log(oracle.accept_uniform(77, b, j))
             assert ok == (j == k)
+
+
+def test_accept_then_resample_output_law_is_the_mixture_of_appendix_a():
+    """Lines 11-22 of Algorithm 1 as one routine: with K = 2 the output law is
+    (1 - p_b^K) P_S + p_b^K Q_K, where Q_2 is known exactly by enumerating S x S; K = 1 reduces to
+    (1 - p_b) P_S + p_b P^ (the single fresh candidate)."""
+    V, members, Z, ctx = _small_world(seed=9)
+    S = oracle.OracleSet(*csr(members), V)
+    logP, logx, P_hat, P_S, PLS = _exact(members, Z, ctx, V)
+    p_b = 1 - PLS
+    x = np.exp(logx)
+    Q = {1: P_hat, 2: 2 * P_hat * (P_hat[None, :] * (x[:, None] / (x[:, None] + x[None, :]))).sum(1)}
+    index = {m: j for j, m in enumerate(members)}
+    n = 200_000
+    for K in (1, 2):
+        o = S.decode_markov(Z, np.full(n, ctx, np.int32), 2 * K, seed=500 + K, n_threads=8)
+        r = oracle.accept_resample(o["logw32"], seed=500 + K)
+        # bookkeeping: accepted column, or a fresh one
+        acc = r["first"] >= 0
+        assert np.array_equal(r["choice"][acc], r["first"][acc])
+        assert np.all((r["choice"][~acc] >= K) & (r["choice"][~acc] < 2 * K))
+        assert abs((~acc).mean() - p_b ** K) < 5 * np.sqrt(p_b ** K * (1 - p_b ** K) / n)
+        pick = o["seq"][np.arange(n), r["choice"], :]
+        emp = np.bincount([index[tuple(s)] for s in pick.tolist()], minlength=len(members)) / n
+        want = (1 - p_b ** K) * P_S + p_b ** K * Q[K]
+        assert abs(want.sum() - 1) < 1e-12
+        floor = 0.5 * np.sqrt(2 / np.pi) * np.sqrt(want * (1 - want) / n).sum()
+        assert tv(emp, want) < 1.3 * floor
+        # the mixture is closer to the target than the plain K-way draw it falls back to
+        assert tv(want, P_S) < tv(Q[K], P_S)
+
+
+def test_accept_then_resample_special_cases():
+    K = 3
+    lw = np.full((4, 2 * K), -1.0, np.float32)
+    lw[0, :K] = 0.0                    # x = 1 > eps always: the first candidate is accepted
+    lw[1, :K] = -np.inf                # x = 0: never accepted, falls back
+    lw[1, K:] = [-np.inf, -2.0, -np.inf]    # only one fresh candidate has weight
+    lw[2, :K] = [-np.inf, 0.0, 0.0]    # the second is the first acceptable one
+    lw[3, :] = -np.inf                 # nothing acceptable, nothing to weigh: uniform fallback, flagged
+    r = oracle.accept_resample(lw, seed=3)
+    assert r["first"].tolist()[:3] == [0, -1, 1] and r["choice"].tolist()[:3] == [0, K + 1, 1]
+    assert r["first"][3] == -1 and K <= r["choice"][3] < 2 * K and r["status"][3] & 2
+    assert abs(r["logz"][1] - (-2.0 - np.log(K))) < 1e-12
