@@ -12,6 +12,8 @@
  *   disc_resample    Algorithm 1, line 22: among K finished candidates pick one with probability
  *                    x_k / sum_j x_j.
  *   disc_accept      Algorithm 1, line 16: accept a candidate when x > eps ~ U[0,1].
+ *   disc_accept_resample  Algorithm 1, lines 11-22: K ordered accept tests, then the K-way draw
+ *                    over K fresh candidates.
  *
  * Conventions
  *   - Every function returns 0 (DISC_OK) or a negative DISC_ERR_* code.  Return codes cover
@@ -211,6 +213,25 @@ int disc_resample(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_
  *               disc_resample on K fresh candidates). */
 int disc_accept(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_t query_base,
                 int32_t* first_out, void* stream);
+
+/* Algorithm 1, lines 11-22 for B queries with 2K finished candidates each: candidates 0..K-1 are
+ * put to the accept test in order (line 16, as disc_accept); the first accepted one is returned;
+ * when all K are rejected, one of the fresh candidates K..2K-1 is drawn with probability
+ * x_k / sum_j x_j (line 22, as disc_resample over those K).  The output then follows
+ * (1 - p_b^K) P_S + p_b^K Q_K (Appendix A), p_b = 1 - P_L(S).
+ *   logw        device, float[B][2K]
+ *   choice_out  device, int32[B]: the candidate returned, in [0, 2K)
+ *   first_out   device, int32[B] (nullable): the accepted candidate, or -1 after K rejections
+ *   logz_out    device, float[B] (nullable): log((1/K) sum x) over the fresh candidates
+ *   seq_tokens  device, int32[B][2K][seq_ld] (nullable) with tokens_out int32[B][seq_ld] (nullable):
+ *               the returned candidate's tokens are copied out
+ *   status_out  device, uint8[B]: status of the K-way draw over the fresh candidates (see
+ *               disc_resample); it matters only where first_out is -1
+ * Random numbers: those of disc_accept and disc_resample for the same seed and query. */
+int disc_accept_resample(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_t query_base,
+                         int32_t* choice_out, int32_t* first_out, float* logz_out,
+                         const int32_t* seq_tokens, int32_t seq_ld, int32_t* tokens_out,
+                         uint8_t* status_out, void* stream);
 
 /* Diagnostic: the n group-noise uniforms of token groups g0 .. g0+n-1 for (seed, step, row), fp32.
  *   out  device, float[n] */

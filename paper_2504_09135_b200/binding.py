@@ -24,7 +24,8 @@ ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "D
           -5: "DISC_ERR_OOM", -6: "DISC_ERR_CUDA", -7: "DISC_ERR_UNSUPPORTED"}
 
 EXPORTS = ["disc_build_set", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
-           "disc_mask", "disc_mask_static", "disc_step", "disc_resample", "disc_accept", "disc_sampling_uniforms",
+           "disc_mask", "disc_mask_static", "disc_step", "disc_resample", "disc_accept", "disc_accept_resample",
+           "disc_sampling_uniforms",
            "disc_error_string", "disc_last_cuda_error"]
 
 
@@ -68,6 +69,7 @@ def lib():
                             vp, vp, i32, vp, vp, vp, vp, vp]
     L.disc_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, i32, vp, vp, vp]
     L.disc_accept.argtypes = [vp, i32, i32, u64, i64, vp, vp]
+    L.disc_accept_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, vp, i32, vp, vp, vp]
     L.disc_sampling_uniforms.argtypes = [u64, u32, u32, i32, i32, vp, vp]
     L.disc_error_string.argtypes = [C.c_int]
     L.disc_error_string.restype = C.c_char_p
@@ -312,6 +314,31 @@ def disc_accept(logw: torch.Tensor, *, seed=0, query_base=0, out=None, stream=No
     rc = lib().disc_accept(_dev(logw, torch.float32, "logw"), B, K, int(seed), int(query_base),
                            _dev(out, torch.int32, "first"), _stream_ptr(stream))
     _check(rc, "disc_accept")
+    return out
+
+
+def disc_accept_resample(logw: torch.Tensor, *, seed=0, query_base=0, seq_tokens: torch.Tensor | None = None,
+                         out=None, stream=None):
+    """logw float32[B, 2K] on the device (first K columns: accept test in order; last K: fresh
+    candidates of the K-way draw) -> dict(choice, first, logz, status, tokens)."""
+    B, K2 = logw.shape
+    if K2 % 2 or K2 == 0:
+        raise DiscError(-1, "disc_accept_resample")
+    dev = logw.device
+    seq_ld = 0 if seq_tokens is None else seq_tokens.shape[-1]
+    if out is None:
+        out = {"choice": torch.empty(B, dtype=torch.int32, device=dev),
+               "first": torch.empty(B, dtype=torch.int32, device=dev),
+               "logz": torch.empty(B, dtype=torch.float32, device=dev),
+               "status": torch.empty(B, dtype=torch.uint8, device=dev),
+               "tokens": None if seq_tokens is None else torch.empty((B, seq_ld), dtype=torch.int32, device=dev)}
+    rc = lib().disc_accept_resample(_dev(logw, torch.float32, "logw"), B, K2 // 2, int(seed), int(query_base),
+                                    _dev(out["choice"], torch.int32, "choice"), _dev(out["first"], torch.int32, "first"),
+                                    _dev(out["logz"], torch.float32, "logz"),
+                                    _dev(seq_tokens, torch.int32, "seq_tokens"), seq_ld,
+                                    _dev(out["tokens"], torch.int32, "tokens"),
+                                    _dev(out["status"], torch.uint8, "status"), _stream_ptr(stream))
+    _check(rc, "disc_accept_resample")
     return out
 
 

@@ -8,7 +8,8 @@ from __future__ import annotations
 
 import torch
 
-from .binding import (DiscSet, DiscState, StepOutputs, disc_resample, disc_state_init, disc_step)
+from .binding import (DiscSet, DiscState, StepOutputs, disc_accept_resample, disc_resample, disc_state_init,
+                      disc_step)
 
 
 class DiscDecoder:
@@ -34,6 +35,15 @@ class DiscDecoder:
     def finish(self, *, seed=0, query_base=0):
         return disc_resample(self.state.logw.view(self.B, self.K), seed=seed, query_base=query_base,
                              seq_tokens=self.seq.view(self.B, self.K, -1), out=self.res)
+
+    def finish_accept_resample(self, *, seed=0, query_base=0):
+        """Algorithm 1, lines 11-22 for a decoder created with an even number of candidates per
+        query: the first half goes through the accept test in order, the second half are the fresh
+        candidates of the K-way draw.  Returns dict(choice, first, logz, status, tokens)."""
+        if self.K % 2:
+            raise ValueError("finish_accept_resample needs an even number of candidates per query")
+        return disc_accept_resample(self.state.logw.view(self.B, self.K), seed=seed, query_base=query_base,
+                                    seq_tokens=self.seq.view(self.B, self.K, -1))
 
     def decode(self, lm, ctx: torch.Tensor, *, seed=0, inv_temperature=1.0, keep_logits=None):
         """Free-running decode: `lm.logits(prev)` gives the [R, V] logits after tokens `prev`.

@@ -292,3 +292,40 @@ def test_resample_and_accept_parity(K):
         k = min(x for x in (first[b], fo[b]) if x >= 0)
         assert abs(float(lw[b, k]) - np.log(oracle.accept_uniform(99, b + 1000, k))) < 1e-5
     assert bad.sum() <= 2
+
+
+@pytest.mark.parametrize("K", [1, 2, 7, 32, 33, 100])
+def test_accept_then_resample_parity(K):
+    """disc_accept_resample (Algorithm 1, lines 11-22 on 2K candidates) against the oracle."""
+    rng = np.random.default_rng(100 + K)
+    B = 3000
+    lw = (rng.standard_normal((B, 2 * K)) * 2 - 2).astype(np.float32)
+    lw[0, :] = -np.inf                 # nothing acceptable, nothing to weigh
+    lw[1, :K] = 0.0                    # the first candidate is always accepted
+    lw[2, :K] = -np.inf
+    lw[2, K:] = -np.inf
+    lw[2, K + K // 2] = -3.0           # a single fresh candidate carries weight
+    lw[3, K:] = np.nan
+    seq = rng.integers(0, 1000, (B, 2 * K, 4)).astype(np.int32)
+    g = disc.disc_accept_resample(torch.as_tensor(lw, device=DEV), seed=7, query_base=50,
+                                  seq_tokens=torch.as_tensor(seq, device=DEV))
+    o = oracle.accept_resample(lw, seed=7, query_ids=np.arange(B) + 50)
+    first, choice = g["first"].cpu().numpy(), g["choice"].cpu().numpy()
+    # accept test: only a log-weight within fp32 rounding of log(eps) may flip
+    flips = np.nonzero(first != o["first"])[0]
+    for b in flips:
+        k = min(x for x in (first[b], o["first"][b]) if x >= 0)
+        assert abs(float(lw[b, k]) - np.log(oracle.accept_uniform(7, b + 50, k))) < 1e-5
+    assert len(flips) <= 2
+    same = first == o["first"]
+    acc = same & (first >= 0)
+    assert np.array_equal(choice[acc], first[acc])
+    rej = same & (first < 0)
+    diff = rej & (choice != o["choice"])
+    assert np.all(o["gap"][diff] < TOL) and np.all(np.abs(choice[diff] - o["choice"][diff]) == 1)
+    assert diff.sum() <= 3
+    assert np.all((choice[rej] >= K) & (choice[rej] < 2 * K))
+    assert (rej.sum() > 0) and (acc.sum() > 0)
+    assert close(g["logz"].cpu().numpy(), o["logz"]).all()
+    assert np.array_equal(g["status"].cpu().numpy(), o["status"])
+    assert np.array_equal(g["tokens"].cpu().numpy(), seq[np.arange(B), choice])
