@@ -4,9 +4,10 @@
 // prefix.
 //
 // One thread block per row.
-//   * Streaming.  Thread t of the block reads the 16-byte vectors t, t+256, t+512, t+768 of every
-//     16 KB chunk of the row with plain read-only vector loads: four independent loads per thread
-//     and four blocks per SM keep some 64 KB per SM in flight, which is what HBM needs.  (A
+//   * Streaming.  The row is read with plain read-only 16-byte loads.  Sparse rows: thread t takes
+//     vectors t, t+128, ... with eight independent loads in flight; dense rows: a 16 KB chunk has
+//     256 slots, slot s owns vectors s, s+256, s+512, s+768 (four loads in flight), and the block
+//     passes over the slots 128 at a time.  Seven blocks per SM keep some 100 KB per SM in flight.  (A
 //     shared-memory ring filled by bulk asynchronous copies was measured slower than this on
 //     the same data, and needed waits that this version does not have.)  Rows that are not
 //     16-byte aligned take a scalar-load path.
@@ -39,11 +40,11 @@
 
 #include "disc_internal.cuh"
 
-// 128 threads per row and 10 blocks per SM (48 registers per thread) measured best on B200: small
-// blocks keep the share of time a block spends outside its streaming loop low, ten of them keep
-// 1280 threads x 64 bytes in flight per SM.
+// 128 threads per row and 7 blocks per SM (72 registers per thread) measured best on B200 for a
+// whole decode: small blocks keep the share of time a block spends outside its streaming loop low,
+// and eight loads in flight per thread (sparse rows) keep a lone row fast when few rows are left.
 #ifndef DISC_MIN_BLOCKS
-#define DISC_MIN_BLOCKS 10
+#define DISC_MIN_BLOCKS 7
 #endif
 
 namespace {
@@ -479,6 +480,37 @@ __device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const Philox
     }
 }
 
+#ifndef DISC_SPARSE_UNROLL
+#define DISC_SPARSE_UNROLL 8
+#endif
+// Sparse rows need only the sum over all logits, so any split of the vectors will do: thread t
+// takes vectors t, t+T, t+2T, ... and keeps DISC_SPARSE_UNROLL loads in flight.
+template <int DT>
+__device__ __forceinline__ void stream_sparse(Acc& a, const RowCtx& r, const char* rowp, int n_groups) {
+    using E = Elem<DT>;
+    constexpr int NP = E::EPV / 2;
+    constexpr int U = DISC_SPARSE_UNROLL;
+    const uint4* row4 = reinterpret_cast<const uint4*>(rowp);
+    const int nvec = n_groups * (GROUP / E::EPV);
+    int i = threadIdx.x;
+    if (i < nvec) {
+        float2 x[NP];
+        E::unpack(__ldg(row4 + i), x);
+        float mx = fmaxf(x[0].x, x[0].y);
+#pragma unroll
+        for (int k = 1; k < NP; ++k) mx = fmaxf(mx, fmaxf(x[k].x, x[k].y));
+        set_reference(a, r, mx);
+    }
+    for (; i + (U - 1) * STEP_THREADS < nvec; i += U * STEP_THREADS) {
+        uint4 raw[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) raw[u] = ld_stream16(row4 + i + u * STEP_THREADS);
+#pragma unroll
+        for (int u = 0; u < U; ++u) consume_vec_sparse<DT>(a, r, raw[u]);
+    }
+    for (; i < nvec; i += STEP_THREADS) consume_vec_sparse<DT>(a, r, ld_stream16(row4 + i));
+}
+
 // groups [g_begin, g_end) of the row read with scalar loads (whole row on the scalar path; the
 // ragged last group on the vector path)
 template <int DT, bool DENSE>
@@ -627,7 +659,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     // ---- stream the row
     if (VEC) {
         if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups);
-        else stream_vec<DT, false>(a, r, p.rk, rowp, gmask, n_vec_groups);
+        else stream_sparse<DT>(a, r, rowp, n_vec_groups);
     }
     if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
     else stream_groups_scalar<DT, false>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
