@@ -274,20 +274,22 @@ __device__ __forceinline__ void consume_vec_sparse(Acc& a, const RowCtx& r, cons
     }
 }
 
-// dense rows: the allowed part of one vector's exponentials; nb = allowed flags of its tokens
+// dense rows: the allowed part of one vector's exponentials; nb = allowed flags of its tokens.
+// tab[f] holds the four flags of nibble f as floats (1 or 0), so that masking is a multiply-add on
+// the packed pipe and costs the same whatever the mask looks like.  (A non-finite exponential times
+// a zero flag gives NaN; such rows have a non-finite full sum as well and are redone by the careful
+// path.)
 template <int NP>
-__device__ __forceinline__ float masked_sum(const float2* e, const float2& t, uint32_t nb) {
-    constexpr uint32_t FULL = (1u << (2 * NP)) - 1u;
-    if (nb == FULL) return t.x + t.y;
-    float s0 = 0.f, s1 = 0.f;
-    if (nb) {
-#pragma unroll
-        for (int i = 0; i < NP; ++i) {
-            s0 += ((nb >> (2 * i)) & 1u) ? e[i].x : 0.f;
-            s1 += ((nb >> (2 * i + 1)) & 1u) ? e[i].y : 0.f;
-        }
+__device__ __forceinline__ float masked_sum(const float2* e, const float4* __restrict__ tab, uint32_t nb) {
+    const float4 m0 = tab[nb & 15u];
+    float2 acc = __fmul2_rn(e[0], make_float2(m0.x, m0.y));
+    acc = __ffma2_rn(e[1], make_float2(m0.z, m0.w), acc);
+    if constexpr (NP == 4) {
+        const float4 m1 = tab[(nb >> 4) & 15u];
+        acc = __ffma2_rn(e[2], make_float2(m1.x, m1.y), acc);
+        acc = __ffma2_rn(e[3], make_float2(m1.z, m1.w), acc);
     }
-    return s0 + s1;
+    return acc.x + acc.y;
 }
 
 // one group given as up to 8 scalars (scalar path, ragged tails, careful use): x[j] for j < nvalid
@@ -385,7 +387,7 @@ __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
 // 256 apart and share a Philox counter.
 template <int DT, bool DENSE>
 __device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp,
-                                           const uint32_t* gmask, int n_groups) {
+                                           const uint32_t* gmask, int n_groups, const float4* tab) {
     using E = Elem<DT>;
     constexpr int EPV = E::EPV;
     constexpr int NP = EPV / 2;
@@ -443,7 +445,7 @@ __device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const Philox
                             float2 e[NP];
                             const float2 t = vec_exp<DT>(a, r, raw[k], e);
                             a.sa = __fadd2_rn(a.sa, t);
-                            tg[j] += masked_sum<NP>(e, t, (bits[j] >> (h * EPV)) & ((1u << EPV) - 1u));
+                            tg[j] += masked_sum<NP>(e, tab, bits[j] >> (h * EPV));
                         }
                     }
                     a.ok2.x += tg[j];
@@ -537,6 +539,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     __shared__ float scratch[STEP_WARPS];
     __shared__ float fin[4];        // (m, s) of the full row and of the valid set
     __shared__ int32_t s_flag, s_tmp;
+    __shared__ __align__(16) float4 flag_tab[16];   // the four bits of a nibble as floats (dense rows)
 
     const int64_t row = blockIdx.x;
     const int tid = threadIdx.x;
@@ -565,6 +568,10 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     }
 
     // dense rows: locate the prebuilt mask row (root, or a heavy node)
+    if (VEC && tid >= 32 && tid < 48) {
+        const int f = tid - 32;
+        flag_tab[f] = make_float4(float(f & 1), float((f >> 1) & 1), float((f >> 2) & 1), float((f >> 3) & 1));
+    }
     if (tid == 0) {
         int32_t h = -2;                                   // -2: not dense
         if (node == 0) h = -1;                            // -1: the root's row
@@ -658,7 +665,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 
     // ---- stream the row
     if (VEC) {
-        if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups);
+        if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups, flag_tab);
         else stream_sparse<DT>(a, r, rowp, n_vec_groups);
     }
     if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
