@@ -60,6 +60,8 @@ def lib():
         L.oracle_rows.restype = None
         L.oracle_mask.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp]
         L.oracle_mask.restype = None
+        L.oracle_verify.argtypes = [vp, vp, i32, vp, i64, vp, i32, vp, vp, vp]
+        L.oracle_verify.restype = None
         L.oracle_step.argtypes = [vp, vp, C.c_int, i64, i64, C.c_float, u64, u32, vp,
                                   vp, i32, vp, vp, vp,
                                   vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
@@ -152,6 +154,25 @@ class OracleSet:
         status = np.empty(n, dtype=np.uint8)
         lib().oracle_mask(self._h, _p(prefix), ld, _p(prefix_len), n, _p(mask), _p(lo), _p(hi), _p(status))
         return mask, lo, hi, status
+
+    def verify(self, prefix, prefix_len, cand, want_mask=True):
+        """Algorithm 2, lines 4-6: validity of M candidate tokens per prefix by binary search in the
+        sorted array.  cand int32[n, M] -> (valid uint8[n, M], row_index int32[n, M], mask or None)."""
+        prefix = _c(prefix, np.int32)
+        if prefix.ndim == 1:
+            prefix = prefix.reshape(1, -1)
+        prefix_len = _c(prefix_len, np.int32).reshape(-1)
+        n = prefix_len.shape[0]
+        if prefix.shape[1] == 0:
+            prefix = np.zeros((n, 1), dtype=np.int32)
+        cand = _c(cand, np.int32).reshape(n, -1)
+        M = cand.shape[1]
+        valid = np.empty((n, M), np.uint8)
+        row_index = np.empty((n, M), np.int32)
+        mask = np.empty((n, self.W), np.uint32) if want_mask else None
+        lib().oracle_verify(self._h, _p(prefix), prefix.shape[1], _p(prefix_len), n, _p(cand), M, _p(valid),
+                            _p(row_index), _p(mask))
+        return valid, row_index, mask
 
     def step(self, logits, dtype, prefix, depth, done=None, *, inv_temperature=1.0, seed=0, step=0,
              row_ids=None, alt_token=None, n_threads=1):

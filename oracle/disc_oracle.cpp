@@ -463,6 +463,44 @@ void oracle_mask(const void* h, const int32_t* prefix, int32_t prefix_ld, const 
     }
 }
 
+// Algorithm 2, lines 4-6, for n partial sequences with M candidate tokens each.  For candidate m of
+// prefix i the row V_m = a + [t_m] is located in the sorted array X by a binary search for the
+// smallest row that is not lexicographically smaller than V_m (index i_m, N when there is none;
+// Section 3.2 "Parallel Verification"); t_m is valid iff V_m is a prefix of X_{i_m}.  valid is
+// [n][M], row_index [n][M], mask [n][W] (line 6: bit t_m set iff valid; nullable).  A candidate
+// outside [0, V) is invalid.
+void oracle_verify(const void* h, const int32_t* prefix, int32_t prefix_ld, const int32_t* prefix_len,
+                   int64_t n, const int32_t* cand, int32_t M, uint8_t* valid, int32_t* row_index,
+                   uint32_t* mask) {
+    const Trie& T = *static_cast<const Trie*>(h);
+    const int64_t N = int64_t(T.sorted_off.size()) - 1;
+    const int64_t W = (T.V + 31) / 32;
+    std::vector<int64_t> rows(N);
+    for (int64_t j = 0; j < N; ++j) rows[j] = j;
+    std::vector<int32_t> Vm;
+    for (int64_t i = 0; i < n; ++i) {
+        if (mask) std::fill(mask + i * W, mask + (i + 1) * W, 0u);
+        for (int32_t m = 0; m < M; ++m) {
+            const int32_t t = cand[i * M + m];
+            Vm.assign(prefix + i * prefix_ld, prefix + i * prefix_ld + prefix_len[i]);
+            Vm.push_back(t);
+            auto it = std::lower_bound(rows.begin(), rows.end(), Vm, [&](int64_t j, const std::vector<int32_t>& v) {
+                return std::lexicographical_compare(T.sorted_tokens.begin() + T.sorted_off[j],
+                                                    T.sorted_tokens.begin() + T.sorted_off[j + 1], v.begin(), v.end());
+            });
+            const int64_t im = it - rows.begin();
+            bool ok = false;
+            if (im < N && t >= 0 && t < T.V) {
+                const int64_t a = T.sorted_off[im], b = T.sorted_off[im + 1];
+                ok = (b - a) >= int64_t(Vm.size()) && std::equal(Vm.begin(), Vm.end(), T.sorted_tokens.begin() + a);
+            }
+            valid[i * M + m] = ok ? 1 : 0;
+            row_index[i * M + m] = int32_t(im);
+            if (ok && mask) mask[i * W + (t >> 5)] |= 1u << (t & 31);
+        }
+    }
+}
+
 // One decoding step for n rows.  Row i's prefix is prefix[i*prefix_ld .. +depth[i]); its logits are
 // logits[i*ld .. +V); its RNG row index is row_ids[i] (i when row_ids is null).  Rows with done[i]
 // != 0 are skipped (token -1, status 8).  Every output array has n entries; alt_token is optional:

@@ -193,3 +193,59 @@ def test_bits_beyond_vocabulary_are_zero():
     mask, *_ = S.mask(np.zeros((1, 2), np.int32), [0])
     assert mask.shape == (1, 2)
     assert int(mask[0, 0]) == 0xFFFFFFFF and int(mask[0, 1]) == (1 << 5) - 1
+
+
+@pytest.mark.parametrize("eos", [False, True])
+def test_verify_candidates_against_a_scan_over_every_member(eos):
+    """Algorithm 2, lines 4-6: a candidate t is valid iff a+[t] is a prefix of some member (scan),
+    the row index is the number of members smaller than a+[t] (Python tuple order), and the
+    extended mask carries exactly the valid candidates."""
+    rng = np.random.default_rng(12 + eos)
+    V, L = 7, 4
+    members = sorted(_random_prefix_free_set(rng, V, L, 60, eos))
+    S = oracle.OracleSet(*_csr(members), V)
+    prefixes = [p for ell in range(0, L) for p in itertools.product(range(V), repeat=ell)]
+    prefixes = [p for p in prefixes if len(p) < 3 or rng.random() < 0.3]
+    n, M = len(prefixes), 5
+    pre = np.zeros((n, L), np.int32)
+    plen = np.array([len(p) for p in prefixes], np.int32)
+    for i, p in enumerate(prefixes):
+        pre[i, :len(p)] = p
+    cand = rng.integers(-1, V + 1, (n, M)).astype(np.int32)      # includes ids outside the vocabulary
+    valid, row_index, mask = S.verify(pre, plen, cand)
+    for i, p in enumerate(prefixes):
+        want_bits = set()
+        for m in range(M):
+            t = int(cand[i, m])
+            vm = tuple(p) + (t,)
+            ok = 0 <= t < V and any(_is_prefix(vm, s) for s in members)
+            assert valid[i, m] == ok, (p, t)
+            assert row_index[i, m] == sum(1 for s in members if s < vm), (p, t)
+            if ok:
+                want_bits.add(t)
+        assert _bits(mask[i], V) == want_bits
+
+
+def test_verify_with_all_tokens_as_candidates_reproduces_the_exact_mask():
+    """With M = |V| (every token a candidate) the verified mask is A_{a,S} itself (Section 3.2,
+    "in theory we should set M = |V|")."""
+    w = scaled("genret", n_draws=3000)
+    tok, off = make_set(w)
+    S = oracle.OracleSet(tok, off, w.V)
+    rng = np.random.default_rng(3)
+    rows = _rows_of(*S.rows())
+    n = 40
+    pre = np.zeros((n, S.l_max), np.int32)
+    plen = np.zeros(n, np.int32)
+    for i in range(n):
+        r = rows[int(rng.integers(0, len(rows)))]
+        d = int(rng.integers(0, len(r)))
+        pre[i, :d] = r[:d]
+        plen[i] = d
+    cand = np.tile(np.arange(w.V, dtype=np.int32), (n, 1))
+    valid, row_index, mask = S.verify(pre, plen, cand)
+    m2, lo, hi, st = S.mask(pre, plen)
+    assert np.array_equal(mask, m2)
+    # the rows the searches land on lie inside the prefix's member range (or right behind it)
+    assert np.all((row_index >= lo[:, None]) & (row_index <= hi[:, None]))
+    assert np.all(row_index[valid == 1] < hi[:, None].repeat(w.V, 1)[valid == 1])
