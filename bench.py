@@ -363,6 +363,27 @@ def run_ours(args):
                        "mask_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                        "frac": round(nbytes / (ms * 1e-3) / 1e9 / peak, 4)}
         del out
+        # top-M verification (Algorithm 2 as stated) of B*K prefixes of the same kind, M = 50 and 500
+        nv = dec.R
+        vrng = np.random.default_rng(7)
+        verify = []
+        for M in (50, 500):
+            cand = torch.as_tensor(vrng.integers(0, w.V, (nv, M)).astype(np.int32), device=dev)
+            vo = disc.disc_verify(G, pre_d[:nv].contiguous(), len_d[:nv].contiguous(), cand)
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(3):
+                disc.disc_verify(G, pre_d[:nv], len_d[:nv], cand, out=vo)
+            a.record()
+            for _ in range(10):
+                disc.disc_verify(G, pre_d[:nv], len_d[:nv], cand, out=vo)
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / 10
+            verify.append({"prefixes": nv, "M": M, "ms": round(ms, 4),
+                           "candidates_per_s": round(nv * M / (ms * 1e-3), 1),
+                           "valid_fraction": round(float(vo["valid"].float().mean().item()), 4)})
+        mask_stress["verify_top_m"] = verify
 
     # ---- CPU baseline: the oracle as it stands, on a bounded sample, rank 0 at N = 1 only
     cpu = None

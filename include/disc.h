@@ -7,6 +7,8 @@
  *                    members of S lexicographically by token id and keep the array on the GPU.
  *   disc_mask        Algorithm 2, lines 3-7 with M = |V|: the mask of the valid set A_{a,S}
  *                    (Section 2.1) of a prefix a.
+ *   disc_verify      Algorithm 2, lines 4-6 as stated: M candidate tokens per prefix verified by
+ *                    binary search in the sorted array (top-M mode).
  *   disc_step        Algorithm 1, lines 5-8 for a batch of partial sequences: mask, sample from
  *                    P.mask/|P.mask|_1, append, multiply the importance score by |P.mask|_1.
  *   disc_resample    Algorithm 1, line 22: among K finished candidates pick one with probability
@@ -164,6 +166,26 @@ int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
 int disc_mask_static(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
                      const int32_t* prefix_len, int64_t n, uint32_t* mask_out, int32_t* lo_out,
                      int32_t* hi_out, int32_t* node_out, uint8_t* status_out, void* stream);
+
+/* Algorithm 2 as stated (lines 4-6; Section 3.2 "Parallel Verification"): for each of n partial
+ * sequences a and each of its M candidate tokens t_m, find by binary search in the sorted member
+ * array X the smallest row that is not lexicographically smaller than V_m = a + [t_m]; t_m is
+ * valid iff V_m is a prefix of that row.  Only the sorted table is read, not the prefix index.
+ *   prefix, prefix_ld, prefix_len   as for disc_mask (0 <= prefix_len[i] <= prefix_ld, at most
+ *               DISC_MAX_DEPTH; a prefix outside that gets the empty range [0, 0))
+ *   cand        device, int32[n][M]: the candidates (for instance the top-M tokens of P); ids
+ *               outside [0, V) are invalid
+ *   valid_out   device, uint8[n][M]: mask_V of Algorithm 2, line 5
+ *   row_out     device, int32[n][M] (nullable): the row index the search lands on (N when every
+ *               row is smaller)
+ *   mask_out    device, uint32[n][W] (nullable): line 6, bit t_m set iff t_m is valid, all other
+ *               bits zero; with every token among the candidates this is disc_mask's mask
+ *   lo_out, hi_out  device, int32[n] (required): the rows having a as a prefix are [lo, hi) (empty
+ *               range with lo = hi = insertion point when there is none)
+ * M = 0 computes the ranges only.  Errors: DISC_ERR_ARG; DISC_ERR_UNSUPPORTED when n*M >= 2^38. */
+int disc_verify(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld, const int32_t* prefix_len,
+                int64_t n, const int32_t* cand, int32_t M, uint8_t* valid_out, int32_t* row_out,
+                uint32_t* mask_out, int32_t* lo_out, int32_t* hi_out, void* stream);
 
 /* One decoding step for n candidates (Algorithm 1, lines 5-8; score closed form in Appendix A).
  *   logits   device, n rows of V values of type `dtype`, row i at element offset i*ld.  The fast

@@ -24,7 +24,7 @@ ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "D
           -5: "DISC_ERR_OOM", -6: "DISC_ERR_CUDA", -7: "DISC_ERR_UNSUPPORTED"}
 
 EXPORTS = ["disc_build_set", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
-           "disc_mask", "disc_mask_static", "disc_step", "disc_resample", "disc_accept", "disc_accept_resample",
+           "disc_mask", "disc_mask_static", "disc_verify", "disc_step", "disc_resample", "disc_accept", "disc_accept_resample",
            "disc_sampling_uniforms",
            "disc_error_string", "disc_last_cuda_error"]
 
@@ -65,6 +65,7 @@ def lib():
     L.disc_state_init.argtypes = [vp, i64, vp, vp, vp, vp, vp, vp, vp]
     L.disc_mask.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp, vp, vp]
     L.disc_mask_static.argtypes = [vp, vp, i32, vp, i64, vp, vp, vp, vp, vp, vp]
+    L.disc_verify.argtypes = [vp, vp, i32, vp, i64, vp, i32, vp, vp, vp, vp, vp, vp]
     L.disc_step.argtypes = [vp, vp, C.c_int, i64, i64, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
                             vp, vp, i32, vp, vp, vp, vp, vp]
     L.disc_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, i32, vp, vp, vp]
@@ -209,6 +210,30 @@ def disc_mask(s: DiscSet, prefix: torch.Tensor, prefix_len: torch.Tensor, *, wan
                          _dev(out["hi"], torch.int32, "hi"), _dev(out["node"], torch.int32, "node"),
                          _dev(out["status"], torch.uint8, "status"), _stream_ptr(stream))
     _check(rc, "disc_mask")
+    return out
+
+
+def disc_verify(s: DiscSet, prefix: torch.Tensor, prefix_len: torch.Tensor, cand: torch.Tensor, *, want_rows=True,
+                want_mask=False, out=None, stream=None):
+    """Algorithm 2, lines 4-6: prefix int32[n, ld], prefix_len int32[n], cand int32[n, M] on the
+    device -> dict(valid uint8[n, M], rows int32[n, M] or None, mask or None, lo, hi)."""
+    n = prefix_len.shape[0]
+    dev = prefix_len.device
+    ld = prefix.shape[1] if prefix.ndim == 2 else 0
+    M = cand.shape[1] if cand.ndim == 2 else 0
+    if out is None:
+        out = {"valid": torch.empty((n, M), dtype=torch.uint8, device=dev),
+               "rows": torch.empty((n, M), dtype=torch.int32, device=dev) if want_rows else None,
+               "mask": torch.empty((n, s.W), dtype=torch.int32, device=dev) if want_mask else None,
+               "lo": torch.empty(n, dtype=torch.int32, device=dev),
+               "hi": torch.empty(n, dtype=torch.int32, device=dev)}
+    rc = lib().disc_verify(s.handle, _dev(prefix, torch.int32, "prefix") if ld > 0 else 0, ld,
+                           _dev(prefix_len, torch.int32, "prefix_len"), n,
+                           _dev(cand, torch.int32, "cand") if M > 0 else 0, M,
+                           _dev(out["valid"], torch.uint8, "valid") if M > 0 else 0,
+                           _dev(out["rows"], torch.int32, "rows"), _dev(out["mask"], torch.int32, "mask"),
+                           _dev(out["lo"], torch.int32, "lo"), _dev(out["hi"], torch.int32, "hi"), _stream_ptr(stream))
+    _check(rc, "disc_verify")
     return out
 
 

@@ -329,3 +329,61 @@ def test_accept_then_resample_parity(K):
     assert close(g["logz"].cpu().numpy(), o["logz"]).all()
     assert np.array_equal(g["status"].cpu().numpy(), o["status"])
     assert np.array_equal(g["tokens"].cpu().numpy(), seq[np.arange(B), choice])
+
+
+@pytest.mark.parametrize("name,over,n,M", [("tiny", {}, 300, 9), ("genret", {}, 1500, 50),
+                                           ("llm", dict(n_draws=200_000), 1500, 50),
+                                           ("large", dict(n_draws=300_000), 1200, 100)])
+def test_verify_parity(name, over, n, M):
+    """disc_verify (Algorithm 2, lines 4-6: binary search in the sorted array) against the oracle:
+    validity, the row every search lands on, the extended mask, the prefix's member range."""
+    w = scaled(name, **over)
+    tok, off, G, S = _both(w)
+    prefix, plen = make_prefixes(w, tok, off, n)
+    rng = np.random.default_rng(17)
+    # complete members, broken prefixes, tokens outside the vocabulary inside a prefix
+    extra = n // 10
+    for j, rr in enumerate(rng.integers(0, off.shape[0] - 1, extra)):
+        L = int(off[rr + 1] - off[rr])
+        prefix[j, :L] = tok[off[rr]:off[rr + 1]]
+        plen[j] = L
+    for j in rng.integers(extra, n, extra):
+        if plen[j] > 0:
+            prefix[j, rng.integers(0, plen[j])] = rng.integers(0, w.V)
+    prefix[n - 1, 0] = w.V + 5
+    plen[n - 1] = max(1, plen[n - 1])
+    # candidates: random ids, ids outside [0, V), and for half of the slots a true child
+    cand = rng.integers(-2, w.V + 2, (n, M)).astype(np.int32)
+    m_true, lo_t, hi_t, st_t = S.mask(prefix, plen)
+    for i in range(n):
+        bits = np.nonzero(np.unpackbits(m_true[i].view(np.uint8), bitorder="little"))[0]
+        if len(bits):
+            k = min(M // 2, len(bits))
+            cand[i, :k] = rng.choice(bits, k, replace=False)
+    g = disc.disc_verify(G, torch.as_tensor(prefix, device=DEV), torch.as_tensor(plen, device=DEV),
+                         torch.as_tensor(cand, device=DEV), want_mask=True)
+    valid, rows, mask = S.verify(prefix, plen, cand)
+    assert np.array_equal(g["valid"].cpu().numpy(), valid)
+    assert np.array_equal(g["rows"].cpu().numpy(), rows)
+    assert np.array_equal(g["mask"].cpu().numpy().view(np.uint32), mask)
+    live = st_t == 0
+    assert np.array_equal(g["lo"].cpu().numpy()[live], lo_t[live]) and np.array_equal(g["hi"].cpu().numpy()[live], hi_t[live])
+    dead = ~live
+    assert np.all(g["lo"].cpu().numpy()[dead] == g["hi"].cpu().numpy()[dead])
+    assert valid.sum() > n and (valid == 0).sum() > n
+
+
+def test_verify_with_every_token_a_candidate_gives_disc_masks_mask():
+    """M = |V|: the verified mask equals the enumerated one (two independent device paths: the
+    sorted table alone against the prefix index)."""
+    w = scaled("genret")
+    tok, off, G, S = _both(w)
+    n = 700
+    prefix, plen = make_prefixes(w, tok, off, n)
+    pre, ln = torch.as_tensor(prefix, device=DEV), torch.as_tensor(plen, device=DEV)
+    cand = torch.arange(w.V, dtype=torch.int32, device=DEV).repeat(n, 1)
+    v = disc.disc_verify(G, pre, ln, cand, want_rows=False, want_mask=True)
+    m = disc.disc_mask(G, pre, ln)
+    assert torch.equal(v["mask"], m["mask"]) and torch.equal(v["lo"], m["lo"]) and torch.equal(v["hi"], m["hi"])
+    r = disc.disc_verify(G, pre, ln, cand[:, :0])           # M = 0: ranges only
+    assert torch.equal(r["lo"], m["lo"]) and torch.equal(r["hi"], m["hi"])
