@@ -275,13 +275,17 @@ def run_ours(args):
     g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler2 = ClockSampler(physical_gpu_index(local_rank))
     sampler2.start()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     g0.record()
-    for _ in range(args.steps):
+    marks[0].record()
+    for k in range(args.steps):
         graph.replay()
+        marks[k + 1].record()
     g1.record()
     barrier()
     clocks_graph = sampler2.stop()
     total_ms = g0.elapsed_time(g1)
+    per_decode_ms = np.array([marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)])
     same_tokens = same_tokens and bool(torch.equal(dec.res["tokens"], first_tokens)) \
         and bool(torch.equal(dec.state.logw, first_logw))
     if world > 1:
@@ -404,6 +408,8 @@ def run_ours(args):
                            "parallelism": f"replicated set, queries sharded over {world} GPU(s), no collective"},
                 "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": gpu_launches,
                 "clocks": clocks_graph,
+                "ms_per_step_median": round(float(np.median(per_decode_ms)), 4),
+                "ms_per_step_best": round(float(per_decode_ms.min()), 4),
                 "timed": "each step = one decode (state init, one disc_step per position, resampling) replayed as "
                          "one CUDA graph",
                 "eager": {"value": round(eager_value, 1), "ms_per_step": round(eager_ms, 4),

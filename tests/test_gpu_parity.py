@@ -387,3 +387,54 @@ def test_verify_with_every_token_a_candidate_gives_disc_masks_mask():
     assert torch.equal(v["mask"], m["mask"]) and torch.equal(v["lo"], m["lo"]) and torch.equal(v["hi"], m["hi"])
     r = disc.disc_verify(G, pre, ln, cand[:, :0])           # M = 0: ranges only
     assert torch.equal(r["lo"], m["lo"]) and torch.equal(r["hi"], m["hi"])
+
+
+def test_edge_shapes_threshold_fanouts_maximum_depth_single_member():
+    """Fan-outs on both sides of the gather/dense switch (1024 and 1025 children), members of the
+    maximum supported length (64 tokens), a set with one member, a batch of one row."""
+    V = 2048 + 7
+    rows = [(0, b, 5) for b in range(1024)] + [(1, b, 5) for b in range(1025)]
+    deep = tuple([2] + [int(x) for x in np.random.default_rng(0).integers(0, V, 62)] + [9])
+    rows += [deep, deep[:-1] + (10,)]
+    tok, off = csr(rows)
+    G = disc.disc_build_set(tok, off, V)
+    S = oracle.OracleSet(tok, off, V)
+    assert G.l_max == 64 and G.n_heavy == 1
+    rng = np.random.default_rng(4)
+    for dtype in (torch.float32, torch.bfloat16):
+        R = 64
+        ls = LockStep(G, S, R, with_mask=True)
+        for t in range(G.l_max):
+            logits = torch.as_tensor((rng.standard_normal((R, V + 1)) * 3).astype(np.float32)).to(dtype).to(DEV)
+            ls.step(logits, t, seed=77)
+        assert bool(ls.state.done.all()) and ls.near_ties <= 2
+        seqs = {tuple(t for t in s if t >= 0) for s in ls.seq.cpu().numpy().tolist()}
+        assert seqs <= set(rows) and any(len(s) == 64 for s in seqs) and any(s[0] == 0 for s in seqs) \
+            and any(s[0] == 1 for s in seqs)
+    # masks of the two threshold nodes and of the deepest prefixes
+    prefix = np.zeros((4, 64), np.int32)
+    plen = np.array([1, 1, 63, 64], np.int32)
+    prefix[1, 0] = 1
+    prefix[2, :63] = deep[:63]
+    prefix[3, :64] = deep
+    g = disc.disc_mask(G, torch.as_tensor(prefix, device=DEV), torch.as_tensor(plen, device=DEV))
+    m, lo, hi, st = S.mask(prefix, plen)
+    assert np.array_equal(g["mask"].cpu().numpy().view(np.uint32), m)
+    assert np.array_equal(g["lo"].cpu().numpy(), lo) and np.array_equal(g["hi"].cpu().numpy(), hi)
+    v = disc.disc_verify(G, torch.as_tensor(prefix, device=DEV), torch.as_tensor(plen, device=DEV),
+                         torch.as_tensor(np.tile(np.array([0, 5, 9, 10, 1023, 1024, 1025], np.int32), (4, 1)), device=DEV))
+    vo, ro, _ = S.verify(prefix, plen, np.tile(np.array([0, 5, 9, 10, 1023, 1024, 1025], np.int32), (4, 1)), want_mask=False)
+    assert np.array_equal(v["valid"].cpu().numpy(), vo) and np.array_equal(v["rows"].cpu().numpy(), ro)
+    G.close()
+
+    # one member, one row: every step is forced, the weight is that token's probability
+    one = [(3, 1, 4, 1, 5)]
+    G1 = disc.disc_build_set(*csr(one), 8)
+    S1 = oracle.OracleSet(*csr(one), 8)
+    ls = LockStep(G1, S1, 1, with_mask=True)
+    for t in range(5):
+        ls.step(torch.as_tensor(rng.standard_normal((1, 8)).astype(np.float32), device=DEV), t, seed=1)
+    assert ls.seq.cpu().numpy().tolist() == [list(one[0])] and bool(ls.state.done.all())
+    r = disc.disc_resample(ls.state.logw.view(1, 1), seed=1)
+    assert r["idx"].item() == 0 and abs(r["logz"].item() - ls.state.logw.item()) < 1e-6
+    G1.close()
