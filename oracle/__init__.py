@@ -106,9 +106,22 @@ class OracleError(RuntimeError):
 class OracleSet:
     """The constraint set as an explicit prefix tree."""
 
-    def __init__(self, tokens, row_offsets, vocab_size):
+    def __init__(self, tokens, row_offsets, vocab_size, eok=None):
+        """eok: for sets in which a member may be a prefix of another (Section 2.1), the
+        end-of-keyword token: every member is closed by it, so that the valid set of a prefix that
+        is itself a member contains eok next to the tokens that extend it."""
         tokens = _c(tokens, np.int32)
         row_offsets = _c(row_offsets, np.int64)
+        if eok is not None:
+            if not 0 <= int(eok) < int(vocab_size) or np.any(tokens == int(eok)):
+                raise OracleError(ERR_TOKEN)
+            rows = [np.append(tokens[row_offsets[i]:row_offsets[i + 1]], np.int32(eok))
+                    for i in range(row_offsets.shape[0] - 1)]
+            if any(r.shape[0] == 1 for r in rows):
+                raise OracleError(ERR_EMPTY)
+            tokens = _c(np.concatenate(rows), np.int32) if rows else tokens
+            row_offsets = np.zeros(len(rows) + 1, np.int64)
+            row_offsets[1:] = np.cumsum([r.shape[0] for r in rows])
         h = C.c_void_p()
         rc = lib().oracle_build(_p(tokens), _p(row_offsets), row_offsets.shape[0] - 1,
                                 int(vocab_size), C.byref(h))

@@ -249,3 +249,43 @@ def test_verify_with_all_tokens_as_candidates_reproduces_the_exact_mask():
     # the rows the searches land on lie inside the prefix's member range (or right behind it)
     assert np.all((row_index >= lo[:, None]) & (row_index <= hi[:, None]))
     assert np.all(row_index[valid == 1] < hi[:, None].repeat(w.V, 1)[valid == 1])
+
+
+def test_end_of_keyword_token_for_sets_with_nested_members():
+    """Section 2.1: the valid set of x is {v : x+[v] is a prefix of a member}, and the
+    end-of-keyword token is valid as well when x itself is a member.  Checked by a scan over the
+    members for every sequence over a small vocabulary; members are nested on purpose."""
+    rng = np.random.default_rng(8)
+    V, EOK, L = 6, 5, 4
+    base = {tuple(int(x) for x in rng.integers(0, V - 1, int(rng.integers(1, L + 1)))) for _ in range(40)}
+    members = sorted(base | {m[:k] for m in list(base)[:12] for k in range(1, len(m))})
+    assert any(a != b and _is_prefix(a, b) for a in members for b in members)
+    with pytest.raises(oracle.OracleError):
+        oracle.OracleSet(*_csr(members), V)                      # not prefix-free as it stands
+    S = oracle.OracleSet(*_csr(members), V, eok=EOK)
+    assert S.N == len(members) and S.l_max == max(len(m) for m in members) + 1
+    seqs = [p for ell in range(0, L + 1) for p in itertools.product(range(V - 1), repeat=ell)]
+    pre = np.zeros((len(seqs), L + 1), np.int32)
+    plen = np.array([len(p) for p in seqs], np.int32)
+    for i, p in enumerate(seqs):
+        pre[i, :len(p)] = p
+    mask, lo, hi, st = S.mask(pre, plen)
+    mset = set(members)
+    for i, x in enumerate(seqs):
+        want = {v for v in range(V - 1) if any(_is_prefix(tuple(x) + (v,), s) for s in members)}
+        if tuple(x) in mset:
+            want.add(EOK)
+        if not want:
+            assert st[i] == 1
+            continue
+        assert st[i] == 0 and _bits(mask[i], V) == want, (x, want)
+        assert hi[i] - lo[i] == sum(_is_prefix(x, s) for s in members)
+    # a member followed by the end-of-keyword token is complete: empty valid set
+    for m in members[:10]:
+        full = np.zeros((1, L + 1), np.int32)
+        full[0, :len(m)] = m
+        full[0, len(m)] = EOK
+        mk, _, _, s1 = S.mask(full, np.array([len(m) + 1], np.int32))
+        assert s1[0] == 0 and not mk.any()
+    with pytest.raises(oracle.OracleError):
+        oracle.OracleSet(*_csr([(1, EOK, 2)]), V, eok=EOK)        # the closing token inside a member
