@@ -110,6 +110,18 @@ typedef struct {
 int disc_build_set(const int32_t* tokens, const int64_t* row_offsets, int64_t n_rows,
                    int32_t vocab_size, uint32_t flags, void* stream, disc_set_t** out);
 
+/* The same build for sets in which a member may be a proper prefix of another member (Section 2.1:
+ * "unless the model generates the end-of-keyword token when x_<t is in S").  Every member is
+ * closed by eok_token (on a host copy; the caller's arrays are not changed), which makes the set
+ * prefix-free, and disc_build_set follows.  Afterwards the valid set of a prefix that is itself a
+ * member contains eok_token next to the tokens that extend it, and a candidate is complete once
+ * it has produced eok_token; sequences returned by disc_step / disc_resample end with it.
+ *   eok_token   in [0, vocab_size); must not occur inside any member (DISC_ERR_TOKEN otherwise)
+ * The longest member may have DISC_MAX_DEPTH - 1 tokens.  Other arguments and errors as for
+ * disc_build_set (DISC_ERR_PREFIX cannot occur). */
+int disc_build_set_eok(const int32_t* tokens, const int64_t* row_offsets, int64_t n_rows,
+                       int32_t vocab_size, int32_t eok_token, void* stream, disc_set_t** out);
+
 /* Release the handle and its device memory.  NULL is allowed. */
 void disc_free_set(disc_set_t* s);
 

@@ -23,7 +23,7 @@ MAX_DEPTH = 64
 ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "DISC_ERR_PREFIX",
           -5: "DISC_ERR_OOM", -6: "DISC_ERR_CUDA", -7: "DISC_ERR_UNSUPPORTED"}
 
-EXPORTS = ["disc_build_set", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
+EXPORTS = ["disc_build_set", "disc_build_set_eok", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
            "disc_mask", "disc_mask_static", "disc_verify", "disc_step", "disc_resample", "disc_accept", "disc_accept_resample",
            "disc_sampling_uniforms",
            "disc_error_string", "disc_last_cuda_error"]
@@ -58,6 +58,7 @@ def lib():
     L = C.CDLL(path)
     vp, i32, i64, u32, u64, f32 = C.c_void_p, C.c_int32, C.c_int64, C.c_uint32, C.c_uint64, C.c_float
     L.disc_build_set.argtypes = [vp, vp, i64, i32, u32, vp, C.POINTER(vp)]
+    L.disc_build_set_eok.argtypes = [vp, vp, i64, i32, i32, vp, C.POINTER(vp)]
     L.disc_free_set.argtypes = [vp]
     L.disc_free_set.restype = None
     L.disc_set_info.argtypes = [vp, C.POINTER(_SetInfo)]
@@ -146,6 +147,24 @@ def disc_build_set(tokens, row_offsets, vocab_size: int, stream=None) -> DiscSet
     rc = lib().disc_build_set(tokens.ctypes.data, row_offsets.ctypes.data, row_offsets.shape[0] - 1,
                               int(vocab_size), 0, _stream_ptr(stream), C.byref(h))
     _check(rc, "disc_build_set")
+    info = _SetInfo()
+    _check(lib().disc_set_info(h, C.byref(info)), "disc_set_info")
+    return DiscSet(h, info)
+
+
+def disc_build_set_eok(tokens, row_offsets, vocab_size: int, eok_token: int, stream=None) -> DiscSet:
+    """Like disc_build_set for sets in which a member may be a prefix of another: every member is
+    closed by `eok_token` (Section 2.1's end-of-keyword token) before the build."""
+    tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+    row_offsets = np.ascontiguousarray(row_offsets, dtype=np.int64)
+    if row_offsets.ndim != 1 or row_offsets.shape[0] < 1:
+        raise DiscError(-1, "disc_build_set_eok")
+    if not torch.cuda.is_available():
+        raise RuntimeError("disc_build_set_eok needs a CUDA device; there is no CPU path")
+    h = C.c_void_p()
+    rc = lib().disc_build_set_eok(tokens.ctypes.data, row_offsets.ctypes.data, row_offsets.shape[0] - 1,
+                                  int(vocab_size), int(eok_token), _stream_ptr(stream), C.byref(h))
+    _check(rc, "disc_build_set_eok")
     info = _SetInfo()
     _check(lib().disc_set_info(h, C.byref(info)), "disc_set_info")
     return DiscSet(h, info)

@@ -9,6 +9,8 @@
 // Sorting and scans use CUB; this code is off the per-step path.
 
 #include <chrono>
+#include <new>
+#include <vector>
 #include <cstring>
 #include <new>
 
@@ -460,6 +462,43 @@ int disc_build_set(const int32_t* tokens, const int64_t* row_offsets, int64_t n_
     S->build_seconds = std::chrono::duration<double>(std::chrono::steady_clock::now() - t0).count();
     *out = S;
     return DISC_OK;
+}
+
+// Sets in which a member may be a proper prefix of another (Section 2.1: when the text generated
+// so far is itself a member, the end-of-keyword token is valid next to the tokens that extend
+// it).  Every member is closed by eok_token on a host copy, which makes the set prefix-free, and
+// the ordinary build follows: the valid set of a prefix that is a member then contains eok_token,
+// and a candidate is complete once it has produced it.
+int disc_build_set_eok(const int32_t* tokens, const int64_t* row_offsets, int64_t n_rows, int32_t vocab_size,
+                       int32_t eok_token, void* stream, disc_set_t** out) {
+    if (!out) return DISC_ERR_ARG;
+    *out = nullptr;
+    if (!tokens || !row_offsets || n_rows < 0 || vocab_size <= 0) return DISC_ERR_ARG;
+    if (eok_token < 0 || eok_token >= vocab_size) return DISC_ERR_TOKEN;
+    if (n_rows == 0) return DISC_ERR_EMPTY;
+    const int64_t E = row_offsets[n_rows] - row_offsets[0];
+    if (E < 0) return DISC_ERR_ARG;
+    std::vector<int32_t> tok;
+    std::vector<int64_t> off;
+    try {
+        tok.reserve(size_t(E + n_rows));
+        off.reserve(size_t(n_rows + 1));
+    } catch (const std::bad_alloc&) {
+        return DISC_ERR_OOM;
+    }
+    off.push_back(0);
+    for (int64_t r = 0; r < n_rows; ++r) {
+        const int64_t a = row_offsets[r], b = row_offsets[r + 1];
+        if (b < a) return DISC_ERR_ARG;
+        if (b == a) return DISC_ERR_EMPTY;
+        for (int64_t i = a; i < b; ++i) {
+            if (tokens[i] == eok_token) return DISC_ERR_TOKEN;     // the closing token must not occur inside a member
+            tok.push_back(tokens[i]);
+        }
+        tok.push_back(eok_token);
+        off.push_back(int64_t(tok.size()));
+    }
+    return disc_build_set(tok.data(), off.data(), n_rows, vocab_size, 0u, stream, out);
 }
 
 void disc_free_set(disc_set_t* s) {

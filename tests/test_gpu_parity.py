@@ -438,3 +438,46 @@ def test_edge_shapes_threshold_fanouts_maximum_depth_single_member():
     r = disc.disc_resample(ls.state.logw.view(1, 1), seed=1)
     assert r["idx"].item() == 0 and abs(r["logz"].item() - ls.state.logw.item()) < 1e-6
     G1.close()
+
+
+def test_nested_members_through_the_end_of_keyword_token():
+    """disc_build_set_eok: members that are prefixes of other members (Section 2.1's EOK rule)."""
+    rng = np.random.default_rng(21)
+    V, EOK = 300, 299
+    base = {tuple(int(x) for x in rng.integers(0, V - 1, int(rng.integers(1, 6)))) for _ in range(4000)}
+    members = sorted(base | {m[:k] for m in list(base)[:800] for k in range(1, len(m))})
+    tok, off = csr(members)
+    with pytest.raises(disc.DiscError):
+        disc.disc_build_set(tok, off, V)
+    G = disc.disc_build_set_eok(tok, off, V, EOK)
+    S = oracle.OracleSet(tok, off, V, eok=EOK)
+    gt, go = disc.disc_set_rows(G)
+    ot, oo = S.rows()
+    assert np.array_equal(gt, ot) and np.array_equal(go, oo) and G.N == len(members)
+    # masks of prefixes that are members, proper prefixes, and complete (member + EOK)
+    n = 600
+    prefix = np.zeros((n, G.l_max), np.int32)
+    plen = np.zeros(n, np.int32)
+    for i in range(n):
+        m = members[int(rng.integers(0, len(members)))]
+        k = int(rng.integers(0, len(m) + 2))
+        seq = (m + (EOK,))[:k]
+        prefix[i, :len(seq)] = seq
+        plen[i] = len(seq)
+    g = disc.disc_mask(G, torch.as_tensor(prefix, device=DEV), torch.as_tensor(plen, device=DEV))
+    m, lo, hi, st = S.mask(prefix, plen)
+    assert np.array_equal(g["mask"].cpu().numpy().view(np.uint32), m) and np.array_equal(g["status"].cpu().numpy(), st)
+    assert np.array_equal(g["lo"].cpu().numpy(), lo) and np.array_equal(g["hi"].cpu().numpy(), hi)
+    # a lock-step decode: every result is a member followed by EOK
+    R = 256
+    ls = LockStep(G, S, R, with_mask=True)
+    for t in range(G.l_max):
+        ls.step(torch.as_tensor((rng.standard_normal((R, V)) * 2).astype(np.float32), device=DEV), t, seed=5)
+    assert bool(ls.state.done.all())
+    mset = set(members)
+    for s in ls.seq.cpu().numpy().tolist():
+        s = [t for t in s if t >= 0]
+        assert s[-1] == EOK and tuple(s[:-1]) in mset
+    with pytest.raises(disc.DiscError):
+        disc.disc_build_set_eok(*csr([(1, EOK, 2)]), V, EOK)
+    G.close()
