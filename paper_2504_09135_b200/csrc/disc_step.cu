@@ -487,8 +487,12 @@ __device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const Philox
 #endif
 // Sparse rows need only the sum over all logits, so any split of the vectors will do: thread t
 // takes vectors t, t+T, t+2T, ... and keeps DISC_SPARSE_UNROLL loads in flight.
-template <int DT>
-__device__ __forceinline__ void stream_sparse(Acc& a, const RowCtx& r, const char* rowp, int n_groups) {
+// `after_first` runs once, right after the first batch of loads has been consumed (or at once if
+// the row is shorter than a batch): the kernel uses it to issue loads whose addresses have arrived
+// in the meantime.
+template <int DT, class Hook>
+__device__ __forceinline__ void stream_sparse(Acc& a, const RowCtx& r, const char* rowp, int n_groups,
+                                              Hook after_first) {
     using E = Elem<DT>;
     constexpr int NP = E::EPV / 2;
     constexpr int U = DISC_SPARSE_UNROLL;
@@ -503,13 +507,16 @@ __device__ __forceinline__ void stream_sparse(Acc& a, const RowCtx& r, const cha
         for (int k = 1; k < NP; ++k) mx = fmaxf(mx, fmaxf(x[k].x, x[k].y));
         set_reference(a, r, mx);
     }
+    bool first = true;
     for (; i + (U - 1) * STEP_THREADS < nvec; i += U * STEP_THREADS) {
         uint4 raw[U];
 #pragma unroll
         for (int u = 0; u < U; ++u) raw[u] = ld_stream16(row4 + i + u * STEP_THREADS);
+        if (first) { after_first(); first = false; }
 #pragma unroll
         for (int u = 0; u < U; ++u) consume_vec_sparse<DT>(a, r, raw[u]);
     }
+    if (first) after_first();
     for (; i < nvec; i += STEP_THREADS) consume_vec_sparse<DT>(a, r, ld_stream16(row4 + i));
 }
 
@@ -545,15 +552,20 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     const int tid = threadIdx.x;
     const int lane = tid & 31, warp = tid >> 5;
 
-    if (p.done[row]) {
+    // The block's time outside its streaming loop is a chain of dependent loads; everything that
+    // does not depend on anything is fetched here, side by side.
+    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
+    const uint8_t was_done = p.done[row];
+    const int32_t node = p.node[row];
+    const int32_t depth_old = tid == 0 ? p.depth[row] : 0, hi_old = tid == 0 ? p.hi[row] : 0;
+    if (was_done) {
         if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_DONE; }
         return;
     }
+    const float x_first_logit = E::load(rowp, 0);
     const int n_groups = (p.V + GROUP - 1) / GROUP;       // the last one may be ragged
     const int n_vec_groups = VEC ? p.V / GROUP : 0;       // whole groups are read with 16-byte loads
-    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * E::SIZE;
 
-    const int32_t node = p.node[row];
     int32_t cb = 0, ce = 0;
     if (node >= 0 && int64_t(node) < p.M) { cb = __ldg(p.child_begin + node); ce = __ldg(p.child_begin + node + 1); }
     const int32_t c = ce - cb;
@@ -585,7 +597,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 
     RowCtx r;
     r.c2 = p.c2; r.inv_t = p.inv_t; r.step = p.step; r.row = uint32_t(p.row_base + uint32_t(row));
-    r.xref = E::load(rowp, 0);
+    r.xref = x_first_logit;
     if (!(fabsf(r.xref) < CUDART_INF_F)) r.xref = 0.f;
 
     Acc a;
@@ -605,15 +617,39 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             }
         }
     }
+    // Loads of the gather path and of the final cursor update that can be issued now and used
+    // after the row has been streamed: this thread's first child; for a row with a single child
+    // (a forced step, the common case deep in the tree) the child's index entries as well.
+    const int32_t v_mine = (!dense && tid < c) ? __ldg(p.node_tok + cb + tid) : -1;
+    float x_mine = 0.f;
+    int32_t only_lo = 0, only_cb = 0, only_ce = 0;
+    if (c == 1 && tid == 0) {
+        only_lo = __ldg(p.node_lo + cb);
+        only_cb = __ldg(p.child_begin + cb);
+        only_ce = __ldg(p.child_begin + cb + 1);
+    }
+
+    // ---- stream the row
+    if (VEC) {
+        if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups, flag_tab);
+        else stream_sparse<DT>(a, r, rowp, n_vec_groups, [&] { if (v_mine >= 0) x_mine = E::load(rowp, v_mine); });
+    } else if (v_mine >= 0) {
+        x_mine = E::load(rowp, v_mine);
+    }
+    if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
+    else stream_groups_scalar<DT, false>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
+
     if (!dense) {
-        // gather path: the few allowed logits are read directly.  Every thread adds its child to
+        // ---- gather path: the few allowed logits are read directly.  Every thread adds its child to
         // the valid-set sum; the thread holding the first child of a group also collects the
         // group's members (at most 8 children), forms the group's exact score and, if that score
         // is the best it has seen, draws the token inside the group right away (stage 2), so that
         // nothing of this is left for the end of the block.
+        // The first child of every thread was fetched before the row was streamed and its logit
+        // while the row was streamed (see above).
         for (int i = tid; i < c; i += STEP_THREADS) {
-            const int32_t v = __ldg(p.node_tok + cb + i);
-            const float x = E::load(rowp, v);
+            const int32_t v = i == tid ? v_mine : __ldg(p.node_tok + cb + i);
+            const float x = i == tid ? x_mine : E::load(rowp, v);
             ms_add(ok, x, p.c2);
             const int32_t G = v >> 3;
             const bool leader = (i == 0) || ((__ldg(p.node_tok + cb + i - 1) >> 3) != G);
@@ -662,14 +698,6 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             }
         }
     }
-
-    // ---- stream the row
-    if (VEC) {
-        if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups, flag_tab);
-        else stream_sparse<DT>(a, r, rowp, n_vec_groups);
-    }
-    if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
-    else stream_groups_scalar<DT, false>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
 
     MS all = a.touched ? MS{a.mref, (a.sa.x + a.sa.y) + (a.sb.x + a.sb.y)} : MS{-CUDART_INF_F, 0.f};
     if (dense) ok = a.touched ? MS{a.mref, a.ok2.x + a.ok2.y} : MS{-CUDART_INF_F, 0.f};
@@ -870,18 +898,23 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             const float xt = E::load(rowp, tok);
             const float logq = f_ok ? (fmaf(xt, p.c2, -K.m) - lg_ok) * LN2_F : (xt * p.c2 - l2_ok) * LN2_F;
             const float logp = f_all ? (fmaf(xt, p.c2, -A.m) - lg_all) * LN2_F : (xt * p.c2 - l2_all) * LN2_F;
-            const int32_t d = p.depth[row];
-            const int32_t hi_old = p.hi[row];
+            const int32_t d = depth_old;
             p.token_out[row] = tok;
             if (p.seq_tokens && d < p.seq_ld) p.seq_tokens[size_t(row) * p.seq_ld + d] = tok;
             if (p.logq_out) p.logq_out[row] = logq;
             if (p.logp_out) p.logp_out[row] = logp;
             p.logw[row] += log_mass;
             p.node[row] = child;
-            p.lo[row] = __ldg(p.node_lo + child);
-            p.hi[row] = (child + 1 < ce) ? __ldg(p.node_lo + child + 1) : hi_old;
+            if (c == 1) {       // fetched before the row was streamed
+                p.lo[row] = only_lo;
+                p.hi[row] = hi_old;
+                p.done[row] = only_cb == only_ce ? 1 : 0;
+            } else {
+                p.lo[row] = __ldg(p.node_lo + child);
+                p.hi[row] = (child + 1 < ce) ? __ldg(p.node_lo + child + 1) : hi_old;
+                p.done[row] = (__ldg(p.child_begin + child) == __ldg(p.child_begin + child + 1)) ? 1 : 0;
+            }
             p.depth[row] = d + 1;
-            p.done[row] = (__ldg(p.child_begin + child) == __ldg(p.child_begin + child + 1)) ? 1 : 0;
             p.status_out[row] = st;
         }
     }
