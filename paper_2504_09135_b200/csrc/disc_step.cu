@@ -652,6 +652,10 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             const float x = i == tid ? x_mine : E::load(rowp, v);
             ms_add(ok, x, p.c2);
             const int32_t G = v >> 3;
+            if (c == 1) {           // a forced step: nothing to draw
+                a.best.score = 0.f; a.best.key = v; a.best.child = cb;
+                break;
+            }
             const bool leader = (i == 0) || ((__ldg(p.node_tok + cb + i - 1) >> 3) != G);
             if (leader) {
                 float xs[GROUP];
@@ -895,7 +899,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             uint8_t st = 0;
             if (!f_all) st |= DISC_ROW_NONFINITE;
             if (!f_ok) st |= DISC_ROW_NOMASS;
-            const float xt = E::load(rowp, tok);
+            const float xt = (c == 1 && !dense) ? x_mine : E::load(rowp, tok);
             const float logq = f_ok ? (fmaf(xt, p.c2, -K.m) - lg_ok) * LN2_F : (xt * p.c2 - l2_ok) * LN2_F;
             const float logp = f_all ? (fmaf(xt, p.c2, -A.m) - lg_all) * LN2_F : (xt * p.c2 - l2_all) * LN2_F;
             const int32_t d = depth_old;
