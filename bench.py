@@ -319,27 +319,42 @@ def run_ours(args):
             h.copy_(l)
         staging = torch.empty_like(logits_steps[0])
         torch.cuda.synchronize()
-        dec.replay_from_host(host, staging, seed=seed)
-        barrier()
         n_e2e = max(1, min(args.steps, 3))
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        wall0 = time.perf_counter()
-        a.record()
-        for _ in range(n_e2e):
-            r = dec.replay_from_host(host, staging, seed=seed)
-        b.record()
-        barrier()
-        wall = time.perf_counter() - wall0
-        e2e_ms = max(a.elapsed_time(b), wall * 1e3)
-        if world > 1:
-            tt = torch.tensor([e2e_ms], device=dev, dtype=torch.float64)
-            dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-            e2e_ms = float(tt.item())
-        assert torch.equal(r["tokens"], first_tokens.cpu())
-        h2d = int(sum(h.numel() * h.element_size() for h in host))
-        d2h = int(sum(v.numel() * v.element_size() for v in r.values()))
-        e2e = {"value": round(world * n_e2e * tokens_per_decode / (e2e_ms * 1e-3), 1), "unit": UNIT,
-               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "decodes": n_e2e}
+
+        def timed_e2e(stage):
+            dec.replay_from_host(host, stage, seed=seed)          # warm-up
+            barrier()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            wall0 = time.perf_counter()
+            a.record()
+            for _ in range(n_e2e):
+                r = dec.replay_from_host(host, stage, seed=seed)
+            b.record()
+            barrier()
+            wall = time.perf_counter() - wall0
+            ms = max(a.elapsed_time(b), wall * 1e3)
+            if world > 1:
+                tt = torch.tensor([ms], device=dev, dtype=torch.float64)
+                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
+                ms = float(tt.item())
+            assert torch.equal(r["tokens"], first_tokens.cpu())
+            return ms, int(sum(v.numel() * v.element_size() for v in r.values()))
+
+        # (a) every position's logits copied to the device, then disc_step; (b) disc_step reads the
+        # pinned host tensors in place, so only the rows that are still live cross PCIe
+        copy_ms, d2h = timed_e2e(staging)
+        inplace_ms, _ = timed_e2e(None)
+        h2d_copy = int(sum(h.numel() * h.element_size() for h in host))
+        h2d_inplace = int(sum(alive) * w.V * esize)
+        tps = lambda ms: round(world * n_e2e * tokens_per_decode / (ms * 1e-3), 1)
+        best_inplace = inplace_ms < copy_ms
+        e2e = {"value": tps(min(copy_ms, inplace_ms)), "unit": UNIT,
+               "h2d_bytes_per_step": h2d_inplace if best_inplace else h2d_copy, "d2h_bytes_per_step": d2h,
+               "decodes": n_e2e,
+               "how": ("disc_step reads the pinned host logits in place (live rows only cross PCIe)" if best_inplace
+                       else "cudaMemcpyAsync of every position's logits into a device buffer, then disc_step"),
+               "copy_then_step": {"value": tps(copy_ms), "h2d_bytes_per_step": h2d_copy},
+               "read_in_place": {"value": tps(inplace_ms), "h2d_bytes_per_step": h2d_inplace}}
         del host, staging
 
     # ---- mask-only stress (secondary figure): 65,536 prefixes of the same table

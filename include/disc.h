@@ -202,7 +202,9 @@ int disc_verify(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld, c
 /* One decoding step for n candidates (Algorithm 1, lines 5-8; score closed form in Appendix A).
  *   logits   device, n rows of V values of type `dtype`, row i at element offset i*ld.  The fast
  *            path needs the base 16-byte aligned and ld*sizeof(value) a multiple of 16; other
- *            layouts take a slower scalar path.
+ *            layouts take a slower scalar path.  Pinned (page-locked, device-accessible) host
+ *            memory is accepted as well: the kernel then reads it in place over PCIe, and rows
+ *            that are already complete are not read at all.
  *   inv_temperature  1/T (Algorithm 1's T), finite and > 0
  *   seed, step, row_base  random-number coordinates (see top of file); `step` must differ between
  *            the steps of one decode

@@ -303,7 +303,9 @@ class StepOutputs:
 def disc_step(s: DiscSet, logits: torch.Tensor, state: DiscState, *, inv_temperature=1.0, seed=0, step=0,
               row_base=0, seq_tokens: torch.Tensor | None = None, out: StepOutputs | None = None,
               stream=None) -> StepOutputs:
-    """logits [n, ld] float32 or bfloat16 on the device (row stride ld >= V, unit element stride)."""
+    """logits [n, ld] float32 or bfloat16 (row stride ld >= V, unit element stride): a device tensor,
+    or a pinned host tensor, which the kernel then reads in place over PCIe (only the rows that are
+    still live are read)."""
     n = state.n
     if logits.dtype == torch.float32:
         dt = DISC_F32
@@ -311,11 +313,12 @@ def disc_step(s: DiscSet, logits: torch.Tensor, state: DiscState, *, inv_tempera
         dt = DISC_BF16
     else:
         raise DiscError(-7, "disc_step")
-    if not (logits.is_cuda and logits.ndim == 2 and logits.shape[0] == n and logits.stride(1) == 1):
-        raise TypeError("logits: expected a CUDA tensor [n, >=V] with unit inner stride")
+    if not ((logits.is_cuda or logits.is_pinned()) and logits.ndim == 2 and logits.shape[0] == n
+            and logits.stride(1) == 1):
+        raise TypeError("logits: expected a CUDA (or pinned host) tensor [n, >=V] with unit inner stride")
     ld = logits.stride(0) if n > 1 else max(logits.shape[1], logits.stride(0))
     if out is None:
-        out = StepOutputs.empty(n, logits.device)
+        out = StepOutputs.empty(n, state.node.device)
     seq_ld = 0
     if seq_tokens is not None:
         seq_ld = seq_tokens.shape[-1]

@@ -79,11 +79,16 @@ class DiscDecoder:
             self.replay(logits_per_step, seed=seed, inv_temperature=inv_temperature)
         return graph
 
-    def replay_from_host(self, host_logits_per_step, staging: torch.Tensor, *, seed=0, inv_temperature=1.0):
-        """Same decode with every step's logits copied from (pinned) host memory first, and the
-        result read back to the host at the end."""
+    def replay_from_host(self, host_logits_per_step, staging: torch.Tensor | None, *, seed=0, inv_temperature=1.0):
+        """Same decode with every step's logits coming from pinned host memory, and the result read
+        back to the host at the end.  With a staging tensor every step's logits are copied to the
+        device first; with staging=None the kernel reads the pinned host memory in place, which
+        moves only the rows that are still live across PCIe."""
         self.reset()
         for t, h in enumerate(host_logits_per_step):
+            if staging is None:
+                self.step(h, t, seed=seed, inv_temperature=inv_temperature)
+                continue
             staging.copy_(h, non_blocking=True)
             self.step(staging, t, seed=seed, inv_temperature=inv_temperature)
         r = self.finish(seed=seed)

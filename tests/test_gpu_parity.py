@@ -481,3 +481,24 @@ def test_nested_members_through_the_end_of_keyword_token():
     with pytest.raises(disc.DiscError):
         disc.disc_build_set_eok(*csr([(1, EOK, 2)]), V, EOK)
     G.close()
+
+
+def test_step_reads_pinned_host_logits_in_place():
+    """The same step with the logits left in pinned host memory gives bit-identical results."""
+    w = scaled("llm", n_draws=50_000, B=4, K=8, d=64)
+    tok, off, G, S = _both(w)
+    rng = np.random.default_rng(2)
+    R = w.R
+    for dtype in (torch.bfloat16, torch.float32):
+        st_a = disc.disc_state_init(G, R, device=DEV)
+        st_b = disc.disc_state_init(G, R, device=DEV)
+        for t in range(3):
+            host = torch.as_tensor((rng.standard_normal((R, w.V)) * 2).astype(np.float32)).to(dtype).pin_memory()
+            oa = disc.disc_step(G, host.to(DEV), st_a, seed=9, step=t)
+            ob = disc.disc_step(G, host, st_b, seed=9, step=t)
+            torch.cuda.synchronize()
+            assert torch.equal(oa.token, ob.token) and torch.equal(oa.logq, ob.logq)
+            assert torch.equal(st_a.logw, st_b.logw) and torch.equal(st_a.node, st_b.node)
+    with pytest.raises(TypeError):
+        disc.disc_step(G, torch.zeros((R, w.V), dtype=torch.float32), st_a, seed=9, step=5)   # pageable host memory
+    G.close()
