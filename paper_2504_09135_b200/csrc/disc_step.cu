@@ -584,14 +584,17 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         const int f = tid - 32;
         flag_tab[f] = make_float4(float(f & 1), float((f >> 1) & 1), float((f >> 2) & 1), float((f >> 3) & 1));
     }
-    if (tid == 0) {
-        int32_t h = -2;                                   // -2: not dense
-        if (node == 0) h = -1;                            // -1: the root's row
-        else if (c > DISC_HEAVY_MIN) { h = heavy_index(p.heavy_nodes, p.n_heavy, node); if (h < 0) h = -2; }
-        s_tmp = h;
+    int32_t hsel = -2;                                    // -2: not dense
+    if (node == 0 || c > DISC_HEAVY_MIN) {                // the same for every thread of the block
+        if (tid == 0) {
+            int32_t h = -2;
+            if (node == 0) h = -1;                        // -1: the root's row
+            else { h = heavy_index(p.heavy_nodes, p.n_heavy, node); if (h < 0) h = -2; }
+            s_tmp = h;
+        }
+        __syncthreads();
+        hsel = s_tmp;
     }
-    __syncthreads();
-    const int32_t hsel = s_tmp;
     const bool dense = hsel != -2;
     const uint32_t* gmask = !dense ? nullptr : (hsel == -1 ? p.root_mask : p.heavy_masks + size_t(hsel) * p.Wp);
 
@@ -707,16 +710,23 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     if (dense) ok = a.touched ? MS{a.mref, a.ok2.x + a.ok2.y} : MS{-CUDART_INF_F, 0.f};
     Best best = a.best;
 
-    // ---- block reduction of (all, ok, best)
+    // ---- block reduction of (all, ok, best).  Inside a warp the (m, s) pairs are brought to the
+    // warp's largest reference first (one exponential per lane), then summed; a lane without
+    // terms (m = -inf) adds zero, a poisoned sum (s = NaN) stays poisoned.
+    {
+        const float M_all = warp_max(all.m), M_ok = warp_max(ok.m);
+        float s_all = (M_all == -CUDART_INF_F) ? 0.f : all.s * exp2f(all.m - M_all);
+        float s_ok = (M_ok == -CUDART_INF_F) ? 0.f : ok.s * exp2f(ok.m - M_ok);
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        MS a2{__shfl_xor_sync(0xffffffffu, all.m, o), __shfl_xor_sync(0xffffffffu, all.s, o)};
-        MS k2{__shfl_xor_sync(0xffffffffu, ok.m, o), __shfl_xor_sync(0xffffffffu, ok.s, o)};
-        Best b2{__shfl_xor_sync(0xffffffffu, best.score, o), __shfl_xor_sync(0xffffffffu, best.key, o),
-                __shfl_xor_sync(0xffffffffu, best.child, o)};
-        all = ms_merge(all, a2);
-        ok = ms_merge(ok, k2);
-        best = best_merge(best, b2);
+        for (int o = 16; o > 0; o >>= 1) {
+            s_all += __shfl_xor_sync(0xffffffffu, s_all, o);
+            s_ok += __shfl_xor_sync(0xffffffffu, s_ok, o);
+            Best b2{__shfl_xor_sync(0xffffffffu, best.score, o), __shfl_xor_sync(0xffffffffu, best.key, o),
+                    __shfl_xor_sync(0xffffffffu, best.child, o)};
+            best = best_merge(best, b2);
+        }
+        all = MS{M_all, s_all};
+        ok = MS{M_ok, s_ok};
     }
     if (lane == 0) {
         red_f[0][warp] = all.m; red_f[1][warp] = all.s; red_f[2][warp] = ok.m; red_f[3][warp] = ok.s;
