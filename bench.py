@@ -172,7 +172,10 @@ def run_ours(args):
         raise SystemExit("bench.py: no CUDA device; the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     dev = torch.device("cuda", local_rank)
-    if world > 1:
+    # under torchrun the process group is used even with one rank, so that a 1-GPU launch goes
+    # through the same barrier / max-over-ranks code as an N-GPU launch
+    use_dist = world > 1 or ("RANK" in os.environ and "MASTER_ADDR" in os.environ)
+    if use_dist:
         dist.init_process_group("nccl", device_id=dev)
     w = workload(args)
     t_setup = time.time()
@@ -229,7 +232,7 @@ def run_ours(args):
     del scratch_logits
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -258,7 +261,7 @@ def run_ours(args):
     total_ms = t0.elapsed_time(t1)
     same_tokens = bool(torch.equal(dec.res["tokens"], first_tokens)) and bool(torch.equal(dec.state.logw, first_logw))
     step_ms = np.array([[ev[k][t][0].elapsed_time(ev[k][t][1]) for t in range(L)] for k in range(args.steps)])
-    if world > 1:
+    if use_dist:
         tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         total_ms = float(tt.item())
@@ -288,7 +291,7 @@ def run_ours(args):
     per_decode_ms = np.array([marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)])
     same_tokens = same_tokens and bool(torch.equal(dec.res["tokens"], first_tokens)) \
         and bool(torch.equal(dec.state.logw, first_logw))
-    if world > 1:
+    if use_dist:
         tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
         dist.all_reduce(tt, op=dist.ReduceOp.MAX)
         total_ms = float(tt.item())
@@ -333,7 +336,7 @@ def run_ours(args):
             barrier()
             wall = time.perf_counter() - wall0
             ms = max(a.elapsed_time(b), wall * 1e3)
-            if world > 1:
+            if use_dist:
                 tt = torch.tensor([ms], device=dev, dtype=torch.float64)
                 dist.all_reduce(tt, op=dist.ReduceOp.MAX)
                 ms = float(tt.item())
@@ -437,7 +440,7 @@ def run_ours(args):
                 "setup_s": round(time.time() - t_setup, 1)}
         print(json.dumps(line))
     G.close()
-    if world > 1:
+    if use_dist:
         dist.destroy_process_group()
 
 
