@@ -61,3 +61,54 @@ def test_tv_to_constrained_target_shrinks_with_k(capsys):
         for K, n, d, f in report:
             print("%36d %8d %14.4f %15.4f" % (K, n, d, f))
     G.close()
+
+
+def test_accept_then_resample_law_through_the_cuda_path():
+    """Algorithm 1, lines 11-22 through disc_step + disc_accept_resample on a small world (V = 8,
+    120 members of length 3, p_b around one half): the output law is (1 - p_b^K) P_S + p_b^K Q_K
+    (Appendix A) with Q_2 known by enumerating S x S, the share of fallbacks is p_b^K, and the mean
+    number of candidates used follows E[k] = (1 - p_b^K)/(1 - p_b) + K p_b^K (Theorem 3.1)."""
+    from helpers import csr
+    rng = np.random.default_rng(5)
+    V0, L = 8, 3
+    members = sorted({tuple(int(t) for t in rng.integers(0, V0, L)) for _ in range(120)})
+    V, ctx = V0 + 1, V0                       # the context token is an extra id that is never produced
+    Z = (rng.standard_normal((V, V)) * 1.5).astype(np.float32)
+    Z[:, ctx] = -1e30
+    G = disc.disc_build_set(*csr(members), V)
+    logP, logx = exact_member_tables(members, Z, ctx, V)
+    PLS = np.exp(logP).sum()
+    p_b = 1 - PLS
+    assert 0.2 < p_b < 0.95
+    P_S = np.exp(logP) / PLS
+    P_hat = np.exp(logP - logx)
+    x = np.exp(logx)
+    Q = {1: P_hat, 2: 2 * P_hat * (P_hat[None, :] * (x[:, None] / (x[:, None] + x[None, :]))).sum(1)}
+    lut = np.full(V ** 3, -1, np.int64)
+    for j, m in enumerate(members):
+        lut[(m[0] * V + m[1]) * V + m[2]] = j
+    Zd = torch.as_tensor(Z, device=DEV)
+    for K, n in [(1, 300_000), (2, 200_000)]:
+        dec = disc.DiscDecoder(G, n, 2 * K, DEV, want_logq=False, want_logp=False)
+        dec.reset()
+        prevtok = torch.full((n * 2 * K,), ctx, dtype=torch.int64, device=DEV)
+        for t in range(G.l_max):
+            o = dec.step(Zd.index_select(0, prevtok), t, seed=77 + K)
+            prevtok = o.token.to(torch.int64)
+        r = dec.finish_accept_resample(seed=77 + K)
+        first = r["first"].cpu().numpy()
+        tokens = r["tokens"].cpu().numpy().astype(np.int64)
+        which = lut[(tokens[:, 0] * V + tokens[:, 1]) * V + tokens[:, 2]]
+        assert which.min() >= 0
+        emp = np.bincount(which, minlength=len(members)) / n
+        want = (1 - p_b ** K) * P_S + p_b ** K * Q[K]
+        floor = 0.5 * np.sqrt(2 / np.pi) * np.sqrt(want * (1 - want) / n).sum()
+        assert tv(emp, want) < 1.3 * floor
+        assert tv(emp, Q[K]) > 2 * floor                 # and it is not the plain K-way law
+        rej = (first < 0).mean()
+        assert abs(rej - p_b ** K) < 5 * np.sqrt(p_b ** K * (1 - p_b ** K) / n)
+        used = np.where(first >= 0, first + 1, 2 * K)
+        want_k = (1 - p_b ** K) / (1 - p_b) + K * p_b ** K
+        assert abs(used.mean() - want_k) < 5 * used.std() / np.sqrt(n), (K, p_b, used.mean(), want_k)
+        del dec
+    G.close()
