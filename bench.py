@@ -316,8 +316,14 @@ def run_ours(args):
 
     # ---- end to end: logits start in pinned host memory, result read back to the host
     e2e = None
+    host = None
     if not args.no_e2e:
-        host = [torch.empty(l.shape, dtype=l.dtype, pin_memory=True) for l in logits_steps]
+        try:
+            host = [torch.empty(l.shape, dtype=l.dtype, pin_memory=True) for l in logits_steps]
+        except RuntimeError as err:          # not enough page-locked memory on this host
+            host = None
+            e2e = {"value": None, "unit": UNIT, "unavailable": f"pinned host buffers: {str(err)[:120]}"}
+    if host is not None:
         for h, l in zip(host, logits_steps):
             h.copy_(l)
         staging = torch.empty_like(logits_steps[0])
