@@ -23,6 +23,8 @@
  *     reported in that row's status byte and never fail the call.
  *   - "host" pointers are ordinary CPU memory, "device" pointers are memory of the current CUDA
  *     device, owned by the caller.  `stream` is a cudaStream_t (NULL = the default stream).
+ *     A handle belongs to the device that was current when it was built; calls that take a
+ *     handle return DISC_ERR_ARG when another device is current.
  *   - Except for disc_build_set / disc_free_set / disc_set_info / disc_set_rows, calls only enqueue
  *     kernels on `stream`: they allocate nothing, do not synchronise the host, and finish in
  *     stream order.

@@ -64,6 +64,13 @@ inline int cuda_fail(cudaError_t e) {
     return e == cudaErrorMemoryAllocation ? DISC_ERR_OOM : DISC_ERR_CUDA;
 }
 
+// the handle's memory lives on the device it was built on: calls with another device current are refused
+inline int check_device(const disc_set* s) {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) return DISC_ERR_CUDA;
+    return dev == s->device ? DISC_OK : DISC_ERR_ARG;
+}
+
 #define DISC_CUDA(call)                                         \
     do {                                                        \
         cudaError_t e__ = (call);                               \

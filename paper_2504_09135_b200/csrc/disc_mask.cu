@@ -316,6 +316,7 @@ extern "C" int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t pre
                          int64_t n, uint32_t* mask_out, int32_t* lo_out, int32_t* hi_out, int32_t* node_out,
                          uint8_t* status_out, void* stream) {
     if (!s || n < 0 || prefix_ld < 0) return DISC_ERR_ARG;
+    if (const int rc = disc::check_device(s)) return rc;
     if (n == 0) return DISC_OK;
     if (!prefix_len || !status_out || (prefix_ld > 0 && !prefix)) return DISC_ERR_ARG;
     if (n >= (int64_t(1) << 31) - 65536) return DISC_ERR_UNSUPPORTED;   // the row counter is 32 bits wide
@@ -387,6 +388,7 @@ extern "C" int disc_mask_static(const disc_set_t* s, const int32_t* prefix, int3
                                 int64_t n, uint32_t* mask_out, int32_t* lo_out, int32_t* hi_out,
                                 int32_t* node_out, uint8_t* status_out, void* stream) {
     if (!s || n < 0 || prefix_ld < 0) return DISC_ERR_ARG;
+    if (const int rc = disc::check_device(s)) return rc;
     if (n == 0) return DISC_OK;
     if (!prefix_len || !status_out || (prefix_ld > 0 && !prefix)) return DISC_ERR_ARG;
     if (n > DISC_MASK_STATIC_MAX_ROWS) return DISC_ERR_UNSUPPORTED;   // beyond what the static counter can hand out

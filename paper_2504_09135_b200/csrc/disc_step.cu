@@ -964,6 +964,7 @@ extern "C" {
 int disc_state_init(const disc_set_t* s, int64_t n, int32_t* node, int32_t* lo, int32_t* hi, int32_t* depth,
                     float* logw, uint8_t* done, void* stream) {
     if (!s || n < 0) return DISC_ERR_ARG;
+    if (const int rc = check_device(s)) return rc;
     if (n == 0) return DISC_OK;
     if (!node || !lo || !hi || !depth || !logw || !done) return DISC_ERR_ARG;
     k_state_init<<<unsigned((n + 255) / 256), 256, 0, static_cast<cudaStream_t>(stream)>>>(
@@ -978,6 +979,7 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
               int32_t seq_ld, float* logq_out, float* logp_out, uint32_t* mask_out, uint8_t* status_out,
               void* stream) {
     if (!s || n < 0 || n >= (int64_t(1) << 31)) return DISC_ERR_ARG;
+    if (const int rc = check_device(s)) return rc;
     if (n == 0) return DISC_OK;
     if (!logits || !node || !lo || !hi || !depth || !logw || !done || !token_out || !status_out) return DISC_ERR_ARG;
     if (ld < s->V || row_base < 0 || (seq_tokens && seq_ld <= 0)) return DISC_ERR_ARG;

@@ -115,6 +115,7 @@ extern "C" int disc_verify(const disc_set_t* s, const int32_t* prefix, int32_t p
                            int64_t n, const int32_t* cand, int32_t M, uint8_t* valid_out, int32_t* row_out,
                            uint32_t* mask_out, int32_t* lo_out, int32_t* hi_out, void* stream) {
     if (!s || n < 0 || prefix_ld < 0 || M < 0) return DISC_ERR_ARG;
+    if (const int rc = disc::check_device(s)) return rc;
     if (n == 0) return DISC_OK;
     if (!prefix_len || !lo_out || !hi_out || (prefix_ld > 0 && !prefix)) return DISC_ERR_ARG;
     if (M > 0 && (!cand || !valid_out)) return DISC_ERR_ARG;
