@@ -379,15 +379,14 @@ __device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
     return v;
 }
 
-// The first n_groups whole groups of the row, read with 16-byte loads.
-// Work split inside a chunk of CHUNK_VECS vectors: a block passes over the chunk's 256 slots,
-// STEP_THREADS at a time.  Sparse rows: slot s takes vectors s, s+256, s+512, s+768.  Dense rows
-// work on groups of 8 tokens: bf16 - the same four vectors (one group each); f32 - groups s and
-// s+256 of the chunk's 512 (two adjacent vectors each).  Either way the groups of one slot are
-// 256 apart and share a Philox counter.
-template <int DT, bool DENSE>
-__device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp,
-                                           const uint32_t* gmask, int n_groups, const float4* tab) {
+// Dense rows: the first n_groups whole groups of the row, read with 16-byte loads.
+// A chunk of CHUNK_VECS vectors has 256 slots and the block passes over them STEP_THREADS at a
+// time.  A slot works on groups of 8 tokens: bf16 - vectors s, s+256, s+512, s+768 of the chunk
+// (one group each); f32 - groups s and s+256 of the chunk's 512 (two adjacent vectors each).
+// Either way the groups of one slot are 256 apart and share a Philox counter.
+template <int DT>
+__device__ __forceinline__ void stream_dense(Acc& a, const RowCtx& r, const PhiloxRoundKeys& rk, const char* rowp,
+                                             const uint32_t* gmask, int n_groups, const float4* tab) {
     using E = Elem<DT>;
     constexpr int EPV = E::EPV;
     constexpr int NP = EPV / 2;
@@ -407,19 +406,16 @@ __device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const Philox
             uint32_t bits[GPT];
             bool have[VPT];
             // vector index inside the chunk of this thread's k-th vector
-            auto vidx = [&](int k) { return DENSE ? ((k / VPG) * SLOTS + slot) * VPG + (k % VPG)
-                                                  : k * SLOTS + slot; };
+            auto vidx = [&](int k) { return ((k / VPG) * SLOTS + slot) * VPG + (k % VPG); };
 #pragma unroll
             for (int k = 0; k < VPT; ++k) {
                 have[k] = FULL || (c * CHUNK_VECS + vidx(k) < nvec);
                 if (have[k]) raw[k] = ld_stream16(row4 + c * CHUNK_VECS + vidx(k));
             }
-            if constexpr (DENSE) {
 #pragma unroll
-                for (int j = 0; j < GPT; ++j) {
-                    const int G = c * GPC + j * SLOTS + slot;
-                    bits[j] = (FULL || G < n_groups) ? uint32_t(__ldg(gbytes + G)) : 0u;
-                }
+            for (int j = 0; j < GPT; ++j) {
+                const int G = c * GPC + j * SLOTS + slot;
+                bits[j] = (FULL || G < n_groups) ? uint32_t(__ldg(gbytes + G)) : 0u;
             }
             if (!a.touched && have[0]) {
                 float2 x[NP];
@@ -429,11 +425,7 @@ __device__ __forceinline__ void stream_vec(Acc& a, const RowCtx& r, const Philox
                 for (int i = 1; i < NP; ++i) mx = fmaxf(mx, fmaxf(x[i].x, x[i].y));
                 set_reference(a, r, mx);
             }
-            if constexpr (!DENSE) {
-#pragma unroll
-                for (int k = 0; k < VPT; ++k)
-                    if (have[k]) consume_vec_sparse<DT>(a, r, raw[k]);
-            } else {
+            {
                 float tg[GPT];
 #pragma unroll
                 for (int j = 0; j < GPT; ++j) {
@@ -634,7 +626,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 
     // ---- stream the row
     if (VEC) {
-        if (dense) stream_vec<DT, true>(a, r, p.rk, rowp, gmask, n_vec_groups, flag_tab);
+        if (dense) stream_dense<DT>(a, r, p.rk, rowp, gmask, n_vec_groups, flag_tab);
         else stream_sparse<DT>(a, r, rowp, n_vec_groups, [&] { if (v_mine >= 0) x_mine = E::load(rowp, v_mine); });
     } else if (v_mine >= 0) {
         x_mine = E::load(rowp, v_mine);
