@@ -48,37 +48,51 @@ struct MaskParams {
     unsigned int* work_counter;   // rows handed out so far by the writer kernel
 };
 
-// index of the child with token t among the sorted children [cb, ce), or -1 (one thread).
-// A walk is a chain of dependent loads, so each round probes eight evenly spaced keys at once
-// (independent loads, one latency) and keeps the ninth of the range that can still hold t: a
-// node with 80,000 children takes 5 rounds instead of the 17 of a binary search.
-__device__ __forceinline__ int32_t find_child(const int32_t* __restrict__ node_tok, int32_t cb, int32_t ce, int32_t t) {
+// The child with token t among the sorted children [cb, ce) of a node (one thread).  A walk is a
+// chain of dependent loads, so each round probes eight evenly spaced keys at once (independent
+// loads, one latency) and keeps the ninth of the range that can still hold t: a node with 80,000
+// children takes 5 rounds instead of the 17 of a binary search.  The walk next needs the child's
+// first member row, its next sibling's, and its own child range: those are fetched for every
+// candidate of the last round together with the candidates' tokens, so that a level of the walk
+// costs one memory latency instead of two.  k = -1 if t is not among the children.
+struct ChildInfo {
+    int32_t k, lo, lo_next, cb, ce;
+};
+__device__ __forceinline__ ChildInfo find_child_info(const int32_t* __restrict__ node_tok,
+                                                     const int32_t* __restrict__ node_lo,
+                                                     const int32_t* __restrict__ child_begin, int32_t cb, int32_t ce,
+                                                     int32_t t) {
     constexpr int P = 8;
     int32_t a = cb, b = ce;                 // the first key >= t, if any, is in [a, b]
     while (b - a > P) {
-        const int32_t s = (b - a + P) / (P + 1);          // >= 1; probe j sits at a + (j+1)*s - 1
+        const int32_t s = (b - a + P) / (P + 1);
         int32_t key[P];
 #pragma unroll
         for (int j = 0; j < P; ++j) {
             const int32_t q = a + (j + 1) * s - 1;
             key[j] = q < b ? __ldg(node_tok + q) : 0x7fffffff;
         }
-        int cnt = 0;                        // probes with key < t form a prefix of the probes
+        int cnt = 0;
 #pragma unroll
         for (int j = 0; j < P; ++j) cnt += key[j] < t ? 1 : 0;
-        const int32_t na = a + cnt * s;                     // one past the last probe below t
-        const int32_t nb = cnt < P ? min(b, a + (cnt + 1) * s - 1) : b;   // the first probe not below t, if any
+        const int32_t na = a + cnt * s;
+        const int32_t nb = cnt < P ? min(b, a + (cnt + 1) * s - 1) : b;
         a = na;
         b = nb;
     }
-    int32_t key[P + 1];
+    int32_t key[P + 1], nlo[P + 2], cbg[P + 2];
 #pragma unroll
     for (int j = 0; j <= P; ++j) key[j] = (a + j < ce) ? __ldg(node_tok + a + j) : 0x7fffffff;
-    int32_t hit = -1;
+#pragma unroll
+    for (int j = 0; j <= P + 1; ++j) {
+        nlo[j] = (a + j < ce) ? __ldg(node_lo + a + j) : 0;
+        cbg[j] = (a + j <= ce) ? __ldg(child_begin + a + j) : 0;
+    }
+    ChildInfo r{-1, 0, 0, 0, 0};
 #pragma unroll
     for (int j = P; j >= 0; --j)
-        if (a + j <= b && key[j] == t) hit = a + j;
-    return hit;
+        if (a + j <= b && key[j] == t) r = ChildInfo{a + j, nlo[j], nlo[j + 1], cbg[j], cbg[j + 1]};
+    return r;
 }
 
 __device__ __forceinline__ void st_stream16(uint4* p, const uint4& v) {
@@ -113,16 +127,28 @@ __global__ void __launch_bounds__(MASK_THREADS) disc_mask_search_kernel(const Ma
     bool ok = (len >= 0 && len <= p.prefix_ld);
     int32_t node = 0, lo = 0, hi = p.N, cb = 0, ce = 0;
     if (ok) { cb = __ldg(p.child_begin); ce = __ldg(p.child_begin + 1); }
+    int32_t t_next = (ok && len > 0) ? pre[0] : 0;
     for (int32_t d = 0; ok && d < len; ++d) {
-        const int32_t t = pre[d];
-        int32_t k = -1;
-        if (t >= 0 && t < p.V) k = (node == 0) ? __ldg(p.root_child + t) : find_child(p.node_tok, cb, ce, t);
-        if (k < 0) { ok = false; break; }
-        lo = __ldg(p.node_lo + k);
-        if (k + 1 < ce) hi = __ldg(p.node_lo + k + 1);
-        node = k;
-        cb = __ldg(p.child_begin + k);
-        ce = __ldg(p.child_begin + k + 1);
+        const int32_t t = t_next;
+        if (d + 1 < len) t_next = pre[d + 1];        // fetched while this level is searched
+        if (t < 0 || t >= p.V) { ok = false; break; }
+        if (node == 0) {
+            const int32_t k = __ldg(p.root_child + t);
+            if (k < 0) { ok = false; break; }
+            lo = __ldg(p.node_lo + k);
+            if (k + 1 < ce) hi = __ldg(p.node_lo + k + 1);
+            node = k;
+            cb = __ldg(p.child_begin + k);
+            ce = __ldg(p.child_begin + k + 1);
+        } else {
+            const ChildInfo c = find_child_info(p.node_tok, p.node_lo, p.child_begin, cb, ce, t);
+            if (c.k < 0) { ok = false; break; }
+            lo = c.lo;
+            if (c.k + 1 < ce) hi = c.lo_next;
+            node = c.k;
+            cb = c.cb;
+            ce = c.ce;
+        }
     }
     if (p.lo_out) p.lo_out[i] = ok ? lo : -1;
     if (p.hi_out) p.hi_out[i] = ok ? hi : -1;
@@ -141,8 +167,17 @@ __global__ void __launch_bounds__(MASK_THREADS) disc_mask_search_kernel(const Ma
     if (!ok) { cb = 0; ce = 0; }
     row[0] = uint32_t(ok ? node : -1); row[1] = uint32_t(cb); row[2] = uint32_t(ce); row[3] = uint32_t(sel);
     if (sel == -2) {
+        // child tokens into the head, twelve loads in flight at a time (a store has to wait for its
+        // load, so one load per store would make this a chain as well)
         const int32_t m = min(ce - cb, HEAD_TOKENS);
-        for (int32_t j = 0; j < m; ++j) row[4 + j] = uint32_t(__ldg(p.node_tok + cb + j));
+        for (int32_t j0 = 0; j0 < m; j0 += 12) {
+            int32_t v[12];
+#pragma unroll
+            for (int u = 0; u < 12; ++u) v[u] = (j0 + u < m) ? __ldg(p.node_tok + cb + j0 + u) : 0;
+#pragma unroll
+            for (int u = 0; u < 12; ++u)
+                if (j0 + u < m) row[4 + j0 + u] = uint32_t(v[u]);
+        }
     }
 }
 
