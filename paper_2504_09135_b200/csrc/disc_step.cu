@@ -417,6 +417,12 @@ __device__ __forceinline__ void stream_dense(Acc& a, const RowCtx& r, const Phil
                 const int G = c * GPC + j * SLOTS + slot;
                 bits[j] = (FULL || G < n_groups) ? uint32_t(__ldg(gbytes + G)) : 0u;
             }
+            // The random words of the slot's groups, computed here and not where they are used: the
+            // integer work then overlaps with the exponentials below.  (Skipping the call when every
+            // group of the slot is hopeless even with the luckiest noise was measured: it almost
+            // never applies, even for very peaked logits, and costs the overlap.)
+            const uint32_t G0 = uint32_t(c * GPC + slot);
+            const uint4 w4 = philox4x32_10(group_slot(G0), r.step, r.row, 0u, rk);
             if (!a.touched && have[0]) {
                 float2 x[NP];
                 E::unpack(raw[0], x);
@@ -442,23 +448,18 @@ __device__ __forceinline__ void stream_dense(Acc& a, const RowCtx& r, const Phil
                     }
                     a.ok2.x += tg[j];
                 }
-                // stage 1 of the sampling for this thread's groups of the chunk: nothing to do if
-                // even the largest possible noise cannot lift any of them above the best score
+                // stage 1 of the sampling for this slot's groups of the chunk.  One test for all of
+                // them first: the largest of the four words gives the smallest w, the largest group
+                // mass the largest right-hand side.
                 float tmax = tg[0];
 #pragma unroll
                 for (int j = 1; j < GPT; ++j) tmax = fmaxf(tmax, tg[j]);
-                if (!(tmax * a.cbound < TWO_M24)) {
-                    const uint32_t G0 = uint32_t(c * GPC + slot);
-                    const uint4 w4 = philox4x32_10(group_slot(G0), r.step, r.row, 0u, rk);
-                    // One test for all groups of the chunk first: the largest of the four words
-                    // gives the smallest w, the largest group mass the largest right-hand side.
-                    const uint32_t wmax = max(max(w4.x, w4.y), max(w4.z, w4.w));
-                    if (!(complement_uniform(wmax) >= tmax * a.cbound)) {
+                const uint32_t wmax = max(max(w4.x, w4.y), max(w4.z, w4.w));
+                if (!(complement_uniform(wmax) >= tmax * a.cbound)) {
 #pragma unroll
-                        for (int j = 0; j < GPT; ++j) {
-                            const uint32_t G = G0 + uint32_t(j * SLOTS);
-                            sample_group(a, tg[j], pick_word(w4, group_word(G)), int32_t(G));
-                        }
+                    for (int j = 0; j < GPT; ++j) {
+                        const uint32_t G = G0 + uint32_t(j * SLOTS);
+                        sample_group(a, tg[j], pick_word(w4, group_word(G)), int32_t(G));
                     }
                 }
                 // a better score found by any lane tightens the whole warp's bound
