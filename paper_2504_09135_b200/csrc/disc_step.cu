@@ -7,15 +7,21 @@
 //   * Streaming.  The row is read with plain read-only 16-byte loads.  Sparse rows: thread t takes
 //     vectors t, t+128, ... with eight independent loads in flight; dense rows: a 16 KB chunk has
 //     256 slots, slot s owns vectors s, s+256, s+512, s+768 (four loads in flight), and the block
-//     passes over the slots 128 at a time.  Seven blocks per SM keep some 100 KB per SM in flight.  (A
-//     shared-memory ring filled by bulk asynchronous copies was measured slower than this on
-//     the same data, and needed waits that this version does not have.)  Rows that are not
-//     16-byte aligned take a scalar-load path.
+//     passes over the slots 128 at a time.  Seven blocks per SM keep some 100 KB per SM in
+//     flight.  (A shared-memory ring filled by bulk asynchronous copies was measured slower than
+//     this on the same data, and needed waits that this version does not have.)  Rows that are
+//     not 16-byte aligned take a scalar-load path.
+//   * Latency.  Outside its streaming loop a block follows a chain of dependent loads (state,
+//     child range, child tokens, their logits; at the end the winner's index entries).  Loads
+//     that depend on nothing are issued first and together; each thread's first child token is
+//     fetched before the streaming loop and its logit during it; the gather work runs after the
+//     loop; a row with a single valid token draws nothing and has its next cursor prefetched.
 //   * Sums.  Each thread accumulates sum 2^(x*c - ref) against its own reference (the maximum of
 //     the first logits it sees), c = log2(e)/T.  Per pair of logits: two unpack operations, one
 //     packed fp32x2 FMA, two ex2 and one packed add.  Partial sums are kept as (m, s) pairs meaning
-//     2^m * s and merged exactly.  All differences are formed between references before any large
-//     value is added, so a common offset of the logits does not cost accuracy.
+//     2^m * s and brought to a common reference before they are added.  All differences are
+//     formed between references before any large value is added, so a common offset of the logits
+//     does not cost accuracy.
 //   * Valid set.  The prefix index gives the row's children as a contiguous list.  Rows with at
 //     most DISC_HEAVY_MIN children gather their few logits directly ("gather path").  Rows with
 //     more have a prebuilt bitmask row in global memory (a few MB in total, L2 resident), read
@@ -29,7 +35,8 @@
 //     mass_G / e^best (times a safety factor) is skipped without taking a logarithm; mass_G is
 //     the already accumulated sum of 2^(x*c - ref) times a per-thread constant.  `best` is the
 //     best score any lane of the warp has seen (shared when a lane improves it).  The four
-//     groups a thread owns in one chunk share one Philox counter.
+//     groups a slot owns in one chunk share one Philox call, issued right after the slot's loads
+//     so that its integer chain overlaps with the load latency and the exponentials.
 //   * A row whose fast sums are not finite, or whose valid mass is so small that terms may have
 //     underflowed against a thread's reference, is redone by a plain two-pass routine with exact
 //     scores ("careful path").
