@@ -502,3 +502,33 @@ def test_step_reads_pinned_host_logits_in_place():
     with pytest.raises(TypeError):
         disc.disc_step(G, torch.zeros((R, w.V), dtype=torch.float32), st_a, seed=9, step=5)   # pageable host memory
     G.close()
+
+
+def test_sharded_calls_with_row_base_equal_one_call():
+    """Query sharding (what N GPUs do): decoding the rows in two calls with row_base / query_base
+    set gives bit-identical tokens, log-weights and resampled indices to one call over all rows."""
+    w = scaled("llm", n_draws=100_000, B=12, K=8, d=64)
+    tok, off, G, S = _both(w)
+    lm = StandInLM(*make_lm_weights(w), w.logits, DEV)
+    ctx = torch.as_tensor(make_contexts(w), device=DEV)
+    R, half = w.R, (w.B // 2) * w.K
+    whole = disc.disc_state_init(G, R, device=DEV)
+    pa = disc.disc_state_init(G, half, device=DEV)
+    pb = disc.disc_state_init(G, R - half, device=DEV)
+    seq = torch.full((R, G.l_max), -1, dtype=torch.int32, device=DEV)
+    seq_a, seq_b = seq[:half].clone(), seq[half:].clone()
+    prev = ctx.to(torch.int64).repeat_interleave(w.K)
+    for t in range(G.l_max):
+        logits = lm.logits(prev)
+        o = disc.disc_step(G, logits, whole, seed=5, step=t, seq_tokens=seq)
+        oa = disc.disc_step(G, logits[:half], pa, seed=5, step=t, row_base=0, seq_tokens=seq_a)
+        ob = disc.disc_step(G, logits[half:], pb, seed=5, step=t, row_base=half, seq_tokens=seq_b)
+        assert torch.equal(o.token, torch.cat([oa.token, ob.token]))
+        prev = torch.where(o.token >= 0, o.token.to(torch.int64), prev)
+    assert torch.equal(whole.logw, torch.cat([pa.logw, pb.logw])) and torch.equal(seq, torch.cat([seq_a, seq_b]))
+    r = disc.disc_resample(whole.logw.view(w.B, w.K), seed=5)
+    ra = disc.disc_resample(pa.logw.view(-1, w.K), seed=5, query_base=0)
+    rb = disc.disc_resample(pb.logw.view(-1, w.K), seed=5, query_base=w.B // 2)
+    assert torch.equal(r["idx"], torch.cat([ra["idx"], rb["idx"]]))
+    assert torch.equal(r["logz"], torch.cat([ra["logz"], rb["logz"]]))
+    G.close()
