@@ -184,9 +184,14 @@ def run_ours(args):
     tok, off = make_set(w)
     G = disc.disc_build_set(tok, off, w.V)
     lm = StandInLM(*make_lm_weights(w), w.logits, dev)
+    # weak scaling: the job has world * B queries, rank r decodes the contiguous block
+    # shard_queries gives it; row / query coordinates of the random numbers stay global
+    from paper_2504_09135_b200.shard import gather_query_results, max_over_ranks, shard_queries, sum_over_ranks
+    q_first, q_count = shard_queries(world * w.B, world, rank)
+    assert q_count == w.B
     ctx = torch.as_tensor(make_contexts(w, salt=rank), device=dev)
-    dec = disc.DiscDecoder(G, w.B, w.K, dev)
-    seed = 250409135 + rank
+    dec = disc.DiscDecoder(G, w.B, w.K, dev, query_base=q_first)
+    seed = 250409135
     L = min(G.l_max, args.positions) if args.positions else G.l_max
     esize = 4 if w.logits == "f32" else 2
 
@@ -215,6 +220,7 @@ def run_ours(args):
     assert args.positions or bool(dec.state.done.all()), "decode did not finish within l_max steps"
     del mask_buf, probe
     tokens_per_decode = int(sum(alive))
+    job_tokens_per_decode = int(sum_over_ranks(tokens_per_decode, dev))      # all ranks' rows
     launches = [t for t in range(L) if alive[t] > 0]
     alg_bytes = [alive[t] * (w.V * esize + 46) + 4 * children[t] for t in range(L)]
 
@@ -261,11 +267,8 @@ def run_ours(args):
     total_ms = t0.elapsed_time(t1)
     same_tokens = bool(torch.equal(dec.res["tokens"], first_tokens)) and bool(torch.equal(dec.state.logw, first_logw))
     step_ms = np.array([[ev[k][t][0].elapsed_time(ev[k][t][1]) for t in range(L)] for k in range(args.steps)])
-    if use_dist:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    eager_value = world * args.steps * tokens_per_decode / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, dev)
+    eager_value = args.steps * job_tokens_per_decode / (total_ms * 1e-3)
     eager_ms = total_ms / args.steps
     gpu_launches = args.steps * (1 + L + 1)      # disc_state_init + L x disc_step + disc_resample
 
@@ -291,12 +294,13 @@ def run_ours(args):
     per_decode_ms = np.array([marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)])
     same_tokens = same_tokens and bool(torch.equal(dec.res["tokens"], first_tokens)) \
         and bool(torch.equal(dec.state.logw, first_logw))
-    if use_dist:
-        tt = torch.tensor([total_ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-        total_ms = float(tt.item())
-    value = world * args.steps * tokens_per_decode / (total_ms * 1e-3)
+    total_ms = max_over_ranks(total_ms, dev)
+    value = args.steps * job_tokens_per_decode / (total_ms * 1e-3)
     del graph
+    # the job's result: every query's chosen sequence, gathered in query order (outside the timed
+    # region; a few KB per rank)
+    job_tokens = gather_query_results(dec.res["tokens"], world * w.B)
+    assert job_tokens.shape[0] == world * w.B
 
     # roofline of the dominant kernel (disc_step): algorithmic bytes / device time, launches with live rows
     kern_ms = float(step_ms[:, launches].sum())
@@ -341,11 +345,7 @@ def run_ours(args):
             b.record()
             barrier()
             wall = time.perf_counter() - wall0
-            ms = max(a.elapsed_time(b), wall * 1e3)
-            if use_dist:
-                tt = torch.tensor([ms], device=dev, dtype=torch.float64)
-                dist.all_reduce(tt, op=dist.ReduceOp.MAX)
-                ms = float(tt.item())
+            ms = max_over_ranks(max(a.elapsed_time(b), wall * 1e3), dev)
             assert torch.equal(r["tokens"], first_tokens.cpu())
             return ms, int(sum(v.numel() * v.element_size() for v in r.values()))
 
@@ -355,7 +355,7 @@ def run_ours(args):
         inplace_ms, _ = timed_e2e(None)
         h2d_copy = int(sum(h.numel() * h.element_size() for h in host))
         h2d_inplace = int(sum(alive) * w.V * esize)
-        tps = lambda ms: round(world * n_e2e * tokens_per_decode / (ms * 1e-3), 1)
+        tps = lambda ms: round(n_e2e * job_tokens_per_decode / (ms * 1e-3), 1)
         best_inplace = inplace_ms < copy_ms
         e2e = {"value": tps(min(copy_ms, inplace_ms)), "unit": UNIT,
                "h2d_bytes_per_step": h2d_inplace if best_inplace else h2d_copy, "d2h_bytes_per_step": d2h,

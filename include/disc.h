@@ -41,7 +41,9 @@
  *       in-group     (G, step, row, 3), word 0
  *       resample     (query, 0, 0, 1), word 0
  *       accept       (query, k, 0, 2), word 0
- *     where `row` / `query` is row_base / query_base plus the index inside the call.
+ *     where `row` / `query` is row_base / query_base plus the index inside the call.  Each is one
+ *     32-bit counter word: row_base + n and query_base + B must not exceed 2^32
+ *     (DISC_ERR_UNSUPPORTED otherwise).
  *   - Sampling draws exactly from P.mask/|P.mask|_1 in two stages.  Tokens are taken in groups of
  *     8 consecutive ids (G = v >> 3).  Stage 1 is Gumbel-max over groups: the group maximising
  *     log(sum of e^{z_v/T} over its allowed tokens) - log(-log u_G) wins (the lowest G on an exact
@@ -112,8 +114,8 @@ typedef struct {
 int disc_build_set(const int32_t* tokens, const int64_t* row_offsets, int64_t n_rows,
                    int32_t vocab_size, uint32_t flags, void* stream, disc_set_t** out);
 
-/* The same build for sets in which a member may be a proper prefix of another member (Section 2.1:
- * "unless the model generates the end-of-keyword token when x_<t is in S").  Every member is
+/* The same build for sets in which a member may be a proper prefix of another member (Section 2.1
+ * lets the model stop at a member by emitting an end-of-keyword token there).  Every member is
  * closed by eok_token (on a host copy; the caller's arrays are not changed), which makes the set
  * prefix-free, and disc_build_set follows.  Afterwards the valid set of a prefix that is itself a
  * member contains eok_token next to the tokens that extend it, and a candidate is complete once
@@ -155,7 +157,7 @@ int disc_state_init(const disc_set_t* s, int64_t n, int32_t* node, int32_t* lo, 
  * With mask_out given, the call keeps a row counter in the set handle: two such calls on the
  * same handle must not run on the device at the same time (calls issued to one stream never do;
  * calls on different streams need an event between them, or a handle each).  n must be below
- * 2^31 - 65536 (DISC_ERR_UNSUPPORTED otherwise). */
+ * 2^31 - 2^20 (DISC_ERR_UNSUPPORTED otherwise). */
 int disc_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld,
               const int32_t* prefix_len, int64_t n, uint32_t* mask_out, int32_t* lo_out,
               int32_t* hi_out, int32_t* node_out, uint8_t* status_out, void* stream);

@@ -66,6 +66,12 @@ def lib():
                                   vp, i32, vp, vp, vp,
                                   vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
         L.oracle_step.restype = None
+        L.oracle_step_plain.argtypes = [vp, vp, C.c_int, i64, i64, C.c_float, u64, u32, vp,
+                                        vp, i32, vp, vp,
+                                        vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
+        L.oracle_step_plain.restype = None
+        L.oracle_plain_uniform.argtypes = [u64, u32, u32]
+        L.oracle_plain_uniform.restype = C.c_double
         L.oracle_resample.argtypes = [vp, i32, i32, u64, vp, vp, vp, vp, vp, vp]
         L.oracle_resample.restype = None
         L.oracle_accept.argtypes = [vp, i32, i32, u64, vp, vp]
@@ -220,6 +226,33 @@ class OracleSet:
                           _p(o["status"]), int(n_threads))
         return o
 
+    def step_plain(self, logits, dtype, prefix, depth, done=None, *, inv_temperature=1.0, seed=0, step=0,
+                   row_ids=None, n_threads=1):
+        """The same step with the plain sampler: inverse CDF over the allowed tokens in ascending id,
+        one uniform per (row, step).  Everything but the token (and logq / logp / range / done, which
+        follow the token) equals step()'s."""
+        depth = _c(depth, np.int32).reshape(-1)
+        n = depth.shape[0]
+        logits = np.ascontiguousarray(logits)
+        assert logits.ndim == 2 and logits.shape[0] == n and logits.shape[1] >= self.V
+        assert logits.dtype == (np.float32 if dtype == F32 else np.uint16)
+        prefix = _c(prefix, np.int32)
+        if prefix.ndim == 1:
+            prefix = prefix.reshape(n, -1)
+        if prefix.shape[1] == 0:
+            prefix = np.zeros((n, 1), dtype=np.int32)
+        done = None if done is None else _c(done, np.uint8)
+        row_ids = None if row_ids is None else _c(row_ids, np.int64)
+        o = {"token": np.empty(n, np.int32), "lo": np.empty(n, np.int32), "hi": np.empty(n, np.int32),
+             "done": np.empty(n, np.uint8), "log_mass": np.empty(n), "lse_all": np.empty(n),
+             "lse_ok": np.empty(n), "logq": np.empty(n), "logp": np.empty(n), "status": np.empty(n, np.uint8)}
+        lib().oracle_step_plain(self._h, _p(logits), int(dtype), logits.shape[1], n, float(inv_temperature),
+                                int(seed), int(step), _p(row_ids), _p(prefix), prefix.shape[1], _p(depth), _p(done),
+                                _p(o["token"]), _p(o["lo"]), _p(o["hi"]), _p(o["done"]), _p(o["log_mass"]),
+                                _p(o["lse_all"]), _p(o["lse_ok"]), _p(o["logq"]), _p(o["logp"]), _p(o["status"]),
+                                int(n_threads))
+        return o
+
     def decode_markov(self, Z, ctx, K, *, inv_temperature=1.0, seed=0, query_base=0, n_threads=1):
         """Free-running SampleCandidate x (B*K) + K-way draw under a Markov LM table Z[V, V]."""
         Z = _c(Z, np.float32)
@@ -289,6 +322,11 @@ def group_uniform(seed, step, row, group):
 def ingroup_uniform(seed, step, row, group):
     """Uniform of the inverse-CDF draw inside the winning group."""
     return lib().oracle_ingroup_uniform(int(seed), int(step), int(row), int(group))
+
+
+def plain_uniform(seed, step, row):
+    """Uniform of the plain inverse-CDF sampler for (row, step)."""
+    return lib().oracle_plain_uniform(int(seed), int(step), int(row))
 
 
 def resample_uniform(seed, query):

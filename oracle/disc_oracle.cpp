@@ -26,10 +26,22 @@
 // Readings where the paper is silent (same list as the design notes):
 //   * S must be prefix-free (fixed length, or every member closed by an EOS
 //     that is an ordinary token); then "a in S" is "the node is a leaf".
-//   * sampling is exact and two-stage: Gumbel-max over groups of 8 consecutive
-//     token ids (group score = log of the group's allowed mass + Gumbel noise,
-//     one Philox4x32-10 uniform per (row, step, group), ties to the lowest
-//     group), then an inverse-CDF draw inside the winning group.
+//   * "sample a token from the distribution" (Algorithm 1, line 7) fixes no
+//     mechanism.  Two exact samplers are stated here:
+//       - oracle_step_plain: the textbook inverse CDF over the allowed tokens in
+//         ascending id with one uniform per (row, step).  It knows nothing of
+//         how any kernel is organised and is the plain statement of line 7;
+//       - oracle_step: two stages - Gumbel-max over groups of 8 consecutive
+//         token ids (group score = log of the group's allowed mass + Gumbel
+//         noise, one Philox4x32-10 uniform per (row, step, group), ties to the
+//         lowest group), then an inverse-CDF draw inside the winning group.
+//         The group size (8 ids = one 16-byte vector of bf16 logits) and the
+//         counter layout of the group noise were taken from the CUDA kernel's
+//         vector width and slot geometry, so that the two sides can be
+//         compared token by token; the law it draws from is the same.
+//     Both are pinned to the exact masked softmax (chi-square) on layouts that
+//     stress the grouping, and every quantity that does not depend on the draw
+//     (lse_all, lse_ok, log_mass, status) comes from one shared routine.
 //   * all floating point here is fp64.
 //
 // Parity pins for these functions live in tests/test_oracle_*.py.  The Philox
@@ -257,6 +269,15 @@ double accept_uniform(uint64_t seed, uint32_t query, uint32_t k) {
     return uniform23(out[0]);
 }
 
+// domain 4: one uniform per (row, step) for the plain inverse-CDF sampler
+double plain_uniform(uint64_t seed, uint32_t step, uint32_t row) {
+    uint32_t ctr[4] = {0u, step, row, 4u};
+    uint32_t key[2] = {uint32_t(seed), uint32_t(seed >> 32)};
+    uint32_t out[4];
+    philox4x32_10(ctr, key, out);
+    return uniform23(out[0]);
+}
+
 double load_logit(const void* base, int dtype, int64_t idx) {
     if (dtype == 0) return double(static_cast<const float*>(base)[idx]);
     uint32_t bits = uint32_t(static_cast<const uint16_t*>(base)[idx]) << 16;   // bf16 -> f32
@@ -295,8 +316,11 @@ struct Lse {
 };
 
 // One decoding step of one row (Algorithm 1, lines 5-8) from the node its prefix reaches.
+// plain = true draws the token with the plain inverse-CDF sampler instead of the two-stage one;
+// nothing else differs.
 StepOut step_row(const Trie& T, int32_t node, const void* logits, int dtype, int64_t base,
-                 double inv_t, uint64_t seed, uint32_t step, uint32_t row, int32_t alt_token) {
+                 double inv_t, uint64_t seed, uint32_t step, uint32_t row, int32_t alt_token,
+                 bool plain = false) {
     StepOut o;
     if (node < 0) { o.status = 1; return o; }                 // prefix not in S
     if (T.first_child[node] < 0) { o.status = 8; o.done = 1; o.lo = T.lo[node]; o.hi = T.hi[node]; return o; }
@@ -339,7 +363,27 @@ StepOut step_row(const Trie& T, int32_t node, const void* logits, int dtype, int
     }
     close_group();
     int32_t best_child = T.first_child[node];                  // lowest id unless a group wins
-    if (!win.empty()) {
+    if (plain) {
+        // Algorithm 1, line 7 as a textbook inverse CDF: weights e^{z_v - max} of the allowed
+        // tokens in ascending id, the smallest token whose inclusive cumulative weight exceeds
+        // u * total.  No groups, one uniform per (row, step).
+        double zmax = NEG_INF, total = 0.0;
+        for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c])
+            zmax = std::max(zmax, load_logit(logits, dtype, base + T.tok[c]) * inv_t);
+        if (std::isfinite(zmax)) {
+            for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c])
+                total += std::exp(load_logit(logits, dtype, base + T.tok[c]) * inv_t - zmax);
+            if (std::isfinite(total) && total > 0.0) {
+                const double target = plain_uniform(seed, step, row) * total;
+                double cum = 0.0;
+                for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c]) {
+                    cum += std::exp(load_logit(logits, dtype, base + T.tok[c]) * inv_t - zmax);
+                    best_child = c;                            // the last allowed token if rounding leaves cum <= target
+                    if (cum > target) break;
+                }
+            }
+        }
+    } else if (!win.empty()) {
         double zmax = NEG_INF, total = 0.0;
         for (const Member& m : win) if (m.z > zmax) zmax = m.z;
         std::vector<double> C(win.size());
@@ -538,6 +582,31 @@ void oracle_step(const void* h, const void* logits, int dtype, int64_t ld, int64
     });
 }
 
+// The same step with the plain sampler (inverse CDF over the allowed tokens, one uniform per row
+// and step; see the top of this file).  Arguments as for oracle_step; the outputs that describe the
+// two-stage draw are absent.
+void oracle_step_plain(const void* h, const void* logits, int dtype, int64_t ld, int64_t n,
+                       float inv_temperature, uint64_t seed, uint32_t step, const int64_t* row_ids,
+                       const int32_t* prefix, int32_t prefix_ld, const int32_t* depth, const uint8_t* done,
+                       int32_t* token, int32_t* lo, int32_t* hi, uint8_t* done_out,
+                       double* log_mass, double* lse_all, double* lse_ok, double* logq, double* logp,
+                       uint8_t* status, int n_threads) {
+    const Trie& T = *static_cast<const Trie*>(h);
+    parallel_rows(n, n_threads, [&](int64_t i) {
+        StepOut o;
+        if (done && done[i]) {
+            o.status = 8; o.done = 1;
+        } else {
+            int32_t node = T.walk(prefix + i * prefix_ld, depth[i]);
+            uint32_t row = uint32_t(row_ids ? row_ids[i] : i);
+            o = step_row(T, node, logits, dtype, i * ld, double(inv_temperature), seed, step, row, -1, true);
+        }
+        token[i] = o.token; lo[i] = o.lo; hi[i] = o.hi; done_out[i] = o.done;
+        log_mass[i] = o.log_mass; lse_all[i] = o.lse_all; lse_ok[i] = o.lse_ok;
+        logq[i] = o.logq; logp[i] = o.logp; status[i] = o.status;
+    });
+}
+
 // K-way importance draw for B queries (Algorithm 1, line 22).  logw is [B][K] fp32 (the bytes the
 // CUDA path holds), widened to fp64 here.  query_ids (nullable) are the RNG query indices.
 // gap[b] = distance of the threshold to the nearest boundary of the chosen interval, as a fraction
@@ -643,6 +712,7 @@ double oracle_group_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t
 double oracle_ingroup_uniform(uint64_t seed, uint32_t step, uint32_t row, uint32_t G) {
     return ingroup_uniform(seed, step, row, G);
 }
+double oracle_plain_uniform(uint64_t seed, uint32_t step, uint32_t row) { return plain_uniform(seed, step, row); }
 double oracle_resample_uniform(uint64_t seed, uint32_t query) { return resample_uniform(seed, query); }
 double oracle_accept_uniform(uint64_t seed, uint32_t query, uint32_t k) { return accept_uniform(seed, query, k); }
 

@@ -158,6 +158,7 @@ int disc_resample(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_
                   float* logz_out, const int32_t* seq_tokens, int32_t seq_ld, int32_t* tokens_out,
                   uint8_t* status_out, void* stream) {
     if (B < 0 || K <= 0 || query_base < 0) return DISC_ERR_ARG;
+    if (query_base + B > (int64_t(1) << 32)) return DISC_ERR_UNSUPPORTED;   // the query coordinate is one 32-bit word
     if (B == 0) return DISC_OK;
     if (!logw || !idx_out || !status_out) return DISC_ERR_ARG;
     if ((seq_tokens || tokens_out) && seq_ld <= 0) return DISC_ERR_ARG;
@@ -172,6 +173,7 @@ int disc_accept_resample(const float* logw, int32_t B, int32_t K, uint64_t seed,
                          int32_t* choice_out, int32_t* first_out, float* logz_out, const int32_t* seq_tokens,
                          int32_t seq_ld, int32_t* tokens_out, uint8_t* status_out, void* stream) {
     if (B < 0 || K <= 0 || K > (1 << 29) || query_base < 0) return DISC_ERR_ARG;
+    if (query_base + B > (int64_t(1) << 32)) return DISC_ERR_UNSUPPORTED;   // the query coordinate is one 32-bit word
     if (B == 0) return DISC_OK;
     if (!logw || !choice_out || !status_out) return DISC_ERR_ARG;
     if ((seq_tokens || tokens_out) && seq_ld <= 0) return DISC_ERR_ARG;
@@ -185,6 +187,7 @@ int disc_accept_resample(const float* logw, int32_t B, int32_t K, uint64_t seed,
 int disc_accept(const float* logw, int32_t B, int32_t K, uint64_t seed, int64_t query_base, int32_t* first_out,
                 void* stream) {
     if (B < 0 || K <= 0 || query_base < 0) return DISC_ERR_ARG;
+    if (query_base + B > (int64_t(1) << 32)) return DISC_ERR_UNSUPPORTED;   // the query coordinate is one 32-bit word
     if (B == 0) return DISC_OK;
     if (!logw || !first_out) return DISC_ERR_ARG;
     disc_accept_kernel<<<(B + 127) / 128, 128, 0, static_cast<cudaStream_t>(stream)>>>(

@@ -985,6 +985,8 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     if (ld < s->V || row_base < 0 || (seq_tokens && seq_ld <= 0)) return DISC_ERR_ARG;
     if (!(inv_temperature > 0.f) || !(inv_temperature <= 3.0e38f)) return DISC_ERR_ARG;
     if (dtype != DISC_F32 && dtype != DISC_BF16) return DISC_ERR_UNSUPPORTED;
+    // the row coordinate of the random numbers is one 32-bit counter word
+    if (row_base + n > (int64_t(1) << 32)) return DISC_ERR_UNSUPPORTED;
 
     StepParams p;
     p.logits = logits; p.ld = ld; p.inv_t = inv_temperature; p.c2 = inv_temperature * LOG2E_F;

@@ -13,8 +13,13 @@ from .binding import (DiscSet, DiscState, StepOutputs, disc_accept_resample, dis
 
 
 class DiscDecoder:
-    def __init__(self, s: DiscSet, B: int, K: int, device="cuda", *, want_logq=True, want_logp=True):
+    def __init__(self, s: DiscSet, B: int, K: int, device="cuda", *, want_logq=True, want_logp=True,
+                 query_base: int = 0):
+        """query_base: global index of this decoder's first query when the queries of a job are
+        sharded over several GPUs (shard.shard_queries); it keeps the random-number coordinates of
+        a row independent of how the job was split."""
         self.set, self.B, self.K, self.R = s, B, K, B * K
+        self.query_base = int(query_base)
         self.device = torch.device(device)
         self.state = DiscState.empty(self.R, self.device)
         self.out = StepOutputs.empty(self.R, self.device, logq=want_logq, logp=want_logp)
@@ -28,20 +33,23 @@ class DiscDecoder:
         self.seq.fill_(-1)
         disc_state_init(self.set, self.R, state=self.state)
 
-    def step(self, logits: torch.Tensor, step: int, *, seed=0, inv_temperature=1.0, row_base=0) -> StepOutputs:
+    def step(self, logits: torch.Tensor, step: int, *, seed=0, inv_temperature=1.0, row_base=None) -> StepOutputs:
+        row_base = self.query_base * self.K if row_base is None else row_base
         return disc_step(self.set, logits, self.state, inv_temperature=inv_temperature, seed=seed, step=step,
                          row_base=row_base, seq_tokens=self.seq, out=self.out)
 
-    def finish(self, *, seed=0, query_base=0):
+    def finish(self, *, seed=0, query_base=None):
+        query_base = self.query_base if query_base is None else query_base
         return disc_resample(self.state.logw.view(self.B, self.K), seed=seed, query_base=query_base,
                              seq_tokens=self.seq.view(self.B, self.K, -1), out=self.res)
 
-    def finish_accept_resample(self, *, seed=0, query_base=0):
+    def finish_accept_resample(self, *, seed=0, query_base=None):
         """Algorithm 1, lines 11-22 for a decoder created with an even number of candidates per
         query: the first half goes through the accept test in order, the second half are the fresh
         candidates of the K-way draw.  Returns dict(choice, first, logz, status, tokens)."""
         if self.K % 2:
             raise ValueError("finish_accept_resample needs an even number of candidates per query")
+        query_base = self.query_base if query_base is None else query_base
         return disc_accept_resample(self.state.logw.view(self.B, self.K), seed=seed, query_base=query_base,
                                     seq_tokens=self.seq.view(self.B, self.K, -1))
 

@@ -1,14 +1,16 @@
-"""Parity at the benchmark's full sizes, in the launch configuration bench.py times:
-|S| = 10 M draws (about 10^8 table entries), V = 128,256, 4,096 bf16 rows per disc_step launch, and
-the 65,536-prefix mask-only stress.  The oracle checks a sample of rows one by one (it needs about
-1.5 ms per row and position); masks and ranges of all prefixes are compared in full."""
+"""Parity at the stated sizes of the workloads, in the launch configuration bench.py times:
+the large one (|S| = 10 M draws, about 10^8 table entries, V = 128,256, 4,096 bf16 rows per
+disc_step launch; the oracle checks a sample of rows one by one, about 1.5 ms per row and position,
+plus every row that sits on a node with a prebuilt mask after the first positions), the 65,536-prefix
+mask-only stress (all masks and ranges compared in full), and the generative-retrieval and
+LLM-vocabulary workloads with every row of every position checked."""
 import numpy as np
 import pytest
 import torch
 
 import oracle
 import paper_2504_09135_b200 as disc
-from gpu_helpers import LockStep
+from gpu_helpers import LockStep, assert_near_ties, close, logits_to_host
 from workloads import CONFIGS, make_contexts, make_lm_weights, make_prefixes, make_set, scaled
 from workloads.standin_lm import StandInLM
 
@@ -42,15 +44,28 @@ def test_full_size_decode_on_sampled_rows(large):
     lw = scaled("large", d=256)                      # same logits law, cheaper stand-in projection
     lm = StandInLM(*make_lm_weights(lw), lw.logits, DEV)
     ctx = torch.as_tensor(make_contexts(w), device=DEV)
-    rows = np.arange(5, w.R, 43)                     # 96 of the 4,096 rows
-    ls = LockStep(G, S, w.R, rows=rows)
+    base_rows = np.arange(5, w.R, 43)                # 96 of the 4,096 rows
+    ls = LockStep(G, S, w.R, rows=base_rows)
     prev = ctx.to(torch.int64).repeat_interleave(w.K)
     seed = 99
+    heavy_seen = []
     for t in range(G.l_max):
         logits = lm.logits(prev)
         assert logits.shape == (w.R, w.V) and logits.dtype == torch.bfloat16
         ls.step(logits, t, seed)
         prev = torch.where(ls.out.token >= 0, ls.out.token.to(torch.int64), prev)
+        # Rows whose prefix now has more than 1,024 valid next tokens take the kernel's prebuilt-mask
+        # path at the next position; below the root that path is otherwise reached by few rows, so
+        # every such row joins the sample for the next step.
+        ls.rows = base_rows
+        if t < 3:
+            seq = ls.seq.cpu().numpy()
+            m, _, _, _ = S.mask(seq, np.full(w.R, t + 1, np.int32))
+            fan = np.unpackbits(m.view(np.uint8), axis=1).sum(1)
+            heavy = np.nonzero(fan > 1024)[0]
+            heavy_seen.append(len(heavy))
+            ls.rows = np.union1d(base_rows, heavy)
+    print(f"rows on a node with more than 1,024 children after positions 0..2: {heavy_seen}")
     assert bool(ls.state.done.all())
     # properties that hold for every row: members only, finite non-positive log-weights
     seq = ls.seq.cpu().numpy()
@@ -81,3 +96,92 @@ def test_full_size_mask_stress(large):
         assert np.array_equal(lo_g[a:a + step], lo) and np.array_equal(hi_g[a:a + step], hi)
         assert np.array_equal(g["mask"][a:a + step].cpu().numpy().view(np.uint32), m)
     assert np.all(st_g == 0)
+
+
+def test_full_size_step_from_nodes_with_prebuilt_masks(large):
+    """One step at the full vocabulary from the prefixes with the largest valid sets below the root
+    (the kernel reads their masks from prebuilt rows), every row checked by the oracle."""
+    w, tok, off, G, S = large
+    st_tok, st_off = S.rows()
+    first = st_tok[st_off[:-1]].astype(np.int64)
+    second = st_tok[st_off[:-1] + 1].astype(np.int64)
+    pair = np.unique(first * w.V + second)
+    fan1 = np.bincount(pair // w.V, minlength=w.V)                  # distinct second tokens per first token
+    top1 = np.argsort(-fan1)[:40]
+    assert fan1[top1[-1]] > 1024
+    third = st_tok[st_off[:-1] + 2].astype(np.int64)
+    tri = np.unique((first * w.V + second) * w.V + third)
+    fan2_keys, fan2 = np.unique(tri // w.V, return_counts=True)     # distinct third tokens per (first, second)
+    top2 = fan2_keys[np.argsort(-fan2)[:8]]
+    n = len(top1) + len(top2)
+    prefix = np.zeros((n, 2), np.int32)
+    depth = np.zeros(n, np.int32)
+    prefix[:len(top1), 0] = top1
+    depth[:len(top1)] = 1
+    prefix[len(top1):, 0] = top2 // w.V
+    prefix[len(top1):, 1] = top2 % w.V
+    depth[len(top1):] = 2
+    rng = np.random.default_rng(17)
+    x = torch.as_tensor((rng.standard_normal((n, w.V)) * 1.5).astype(np.float32)).to(torch.bfloat16).to(DEV)
+    pre, dep = torch.as_tensor(prefix, device=DEV), torch.as_tensor(depth, device=DEV)
+    cur = disc.disc_mask(G, pre, dep, want_mask=False)
+    state = disc.DiscState(cur["node"].clone(), cur["lo"].clone(), cur["hi"].clone(), dep.clone(),
+                           torch.zeros(n, dtype=torch.float32, device=DEV), torch.zeros(n, dtype=torch.uint8, device=DEV))
+    out = disc.StepOutputs.empty(n, DEV, mask_words=G.W)
+    disc.disc_step(G, x, state, seed=31, step=2, out=out)
+    torch.cuda.synchronize()
+    hl, dt = logits_to_host(x)
+    o = S.step(hl, dt, prefix, depth, seed=31, step=2, alt_token=out.token.cpu().numpy(), n_threads=8)
+    m, lo, hi, s0 = S.mask(prefix, depth)
+    assert np.array_equal(out.mask.cpu().numpy().view(np.uint32), m)
+    assert np.all(o["n_children"][:len(top1)] > 1024)
+    assert np.array_equal(out.status.cpu().numpy(), o["status"])
+    g_tok = out.token.cpu().numpy()
+    same = g_tok == o["token"]
+    ties = assert_near_ties(g_tok[~same], o, ~same)
+    assert close(state.logw.cpu().numpy(), o["log_mass"]).all()
+    assert close(out.logq.cpu().numpy()[same], o["logq"][same]).all()
+    assert close(out.logp.cpu().numpy()[same], o["logp"][same]).all()
+    assert np.array_equal(state.lo.cpu().numpy()[same], o["lo"][same])
+    assert np.array_equal(state.hi.cpu().numpy()[same], o["hi"][same])
+    assert np.array_equal(state.done.cpu().numpy()[same], o["done"][same])
+    print(f"prebuilt-mask rows checked: {n} (fan-out {int(o['n_children'].min())}..{int(o['n_children'].max())}), "
+          f"near-ties {ties}")
+    assert ties <= 1
+
+
+@pytest.mark.parametrize("name", ["genret", "llm"])
+def test_stated_size_decode_every_row(name):
+    """The generative-retrieval workload (V = 256, 100,000 members, B = 256, K = 8) and the
+    LLM-vocabulary workload (V = 32,000, 1 M draws, B = 64, K = 16, d = 1024) at their stated sizes:
+    every row of every position in lock-step with the oracle, then the K-way draw."""
+    w = CONFIGS[name]
+    tok, off = make_set(w)
+    G = disc.disc_build_set(tok, off, w.V)
+    S = oracle.OracleSet(tok, off, w.V)
+    try:
+        lm = StandInLM(*make_lm_weights(w), w.logits, DEV)
+        ctx = torch.as_tensor(make_contexts(w), device=DEV)
+        ls = LockStep(G, S, w.R, with_mask=True)
+        prev = ctx.to(torch.int64).repeat_interleave(w.K)
+        seed = 20250409 + w.index
+        for t in range(G.l_max):
+            logits = lm.logits(prev)
+            assert logits.shape == (w.R, w.V)
+            ls.step(logits, t, seed)
+            prev = torch.where(ls.out.token >= 0, ls.out.token.to(torch.int64), prev)
+        assert bool(ls.state.done.all())
+        logw = ls.state.logw.view(w.B, w.K)
+        r = disc.disc_resample(logw, seed=seed, seq_tokens=ls.seq.view(w.B, w.K, -1))
+        o = oracle.resample(logw.cpu().numpy(), seed=seed)
+        idx = r["idx"].cpu().numpy()
+        diff = idx != o["idx"]
+        assert np.all(o["gap"][diff] < 1e-5) and np.all(np.abs(idx[diff] - o["idx"][diff]) == 1)
+        assert close(r["logz"].cpu().numpy(), o["logz"]).all()
+        print(f"[{name} at its stated size] rows*positions checked={ls.checked} near-ties={ls.near_ties} "
+              f"resample near-ties={int(diff.sum())} max rel logw err={ls.max_err:.2e}")
+        assert ls.checked == w.R * G.l_max
+        assert ls.near_ties <= max(2, ls.checked // 1000)
+    finally:
+        G.close()
+        S.close()

@@ -8,7 +8,7 @@ import torch
 import torch.distributed as dist
 import torch.multiprocessing as mp
 
-from paper_2504_09135_b200.shard import gather_query_results, max_over_ranks, shard_queries
+from paper_2504_09135_b200.shard import gather_query_results, max_over_ranks, shard_queries, sum_over_ranks
 
 
 def test_shards_tile_the_queries():
@@ -34,7 +34,8 @@ def _worker(rank, world, port, B, q):
         local = torch.arange(start, start + n, dtype=torch.int32).unsqueeze(1).repeat(1, 3) * 10 + rank
         full = gather_query_results(local, B)
         slow = max_over_ranks(1.0 + rank)
-        q.put((rank, full.tolist(), slow))
+        total = sum_over_ranks(10.0 + rank)
+        q.put((rank, full.tolist(), slow, total))
     finally:
         dist.destroy_process_group()
 
@@ -57,6 +58,7 @@ def test_two_ranks_gather_in_query_order():
     for r in range(world):
         s0, n = shard_queries(B, world, r)
         want += [[i * 10 + r] * 3 for i in range(s0, s0 + n)]
-    for rank, full, slow in got:
+    for rank, full, slow, total in got:
         assert full == want
         assert slow == 2.0
+        assert total == 21.0

@@ -1,4 +1,5 @@
-"""disc_mask_static (the entry point that allocates nothing) against disc_mask, through the C ABI.
+"""disc_mask_static (the entry point that allocates nothing) against disc_mask and against the CPU
+oracle, through the C ABI.
 
 Named so that it is collected after the other GPU tests: it must pass both alone and with whatever
 the earlier tests left on the device and in the library's static word block."""
@@ -6,6 +7,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from workloads import make_prefixes, make_set, scaled
 
 pytestmark = pytest.mark.gpu
@@ -48,13 +50,30 @@ def test_static_entry_point_matches_disc_mask_on_two_calls_in_a_row(name, over, 
         for ref, out, pre, ln in pairs:
             disc.disc_mask_static(G, pre, ln, out=out)
         torch.cuda.synchronize()
-        for ref, out, _, _ in pairs:
+        S = oracle.OracleSet(tok, off, w.V)
+        for ref, out, pre, ln in pairs:
             for key in ("mask", "lo", "hi", "node", "status"):
                 assert torch.equal(ref[key], out[key]), key
+            # and against the oracle's prefix tree, so that a fault common to both CUDA entry
+            # points cannot pass
+            m, lo, hi, st = S.mask(pre.cpu().numpy(), ln.cpu().numpy())
+            assert np.array_equal(out["mask"].cpu().numpy().view(np.uint32), m)
+            assert np.array_equal(out["lo"].cpu().numpy(), lo) and np.array_equal(out["hi"].cpu().numpy(), hi)
+            assert np.array_equal(out["status"].cpu().numpy(), st)
+        S.close()
         # ranges only (no mask output) go through the same entry point
         ref, _, pre, ln = pairs[0]
         r2 = disc.disc_mask_static(G, pre, ln, want_mask=False)
         assert r2["mask"] is None and torch.equal(r2["lo"], ref["lo"]) and torch.equal(r2["status"], ref["status"])
+        # the promise of the entry point: with the outputs preallocated, a call takes no device memory
+        ref, out, pre, ln = pairs[1]
+        torch.cuda.synchronize()
+        free_before, _ = torch.cuda.mem_get_info()
+        for _ in range(2):
+            disc.disc_mask_static(G, pre, ln, out=out)
+        torch.cuda.synchronize()
+        free_after, _ = torch.cuda.mem_get_info()
+        assert free_after == free_before
     finally:
         G.close()
 
