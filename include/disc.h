@@ -11,6 +11,9 @@
  *                    binary search in the sorted array (top-M mode).
  *   disc_step        Algorithm 1, lines 5-8 for a batch of partial sequences: mask, sample from
  *                    P.mask/|P.mask|_1, append, multiply the importance score by |P.mask|_1.
+ *   disc_project_step  the same step with line 5's P = L(a, T) folded in: the model's last projection
+ *                    (hidden vectors times the vocabulary matrix) runs on the tensor cores and
+ *                    only the pieces of the logits the step looks at ever reach memory.
  *   disc_resample    Algorithm 1, line 22: among K finished candidates pick one with probability
  *                    x_k / sum_j x_j.
  *   disc_accept      Algorithm 1, line 16: accept a candidate when x > eps ~ U[0,1].
@@ -74,8 +77,9 @@ extern "C" {
 #define DISC_ROW_NOMASS 2   /* allowed probability mass is zero or not finite                     */
 #define DISC_ROW_NONFINITE 4 /* NaN or +Inf among the row's logits (or NaN among the weights)     */
 #define DISC_ROW_DONE 8     /* row was already complete: nothing read, state untouched            */
-#define DISC_ROW_FAULT 16   /* reserved for kernels that wait on asynchronous copies; the present ones
-                               have no waits and never set it                                     */
+#define DISC_ROW_FAULT 16   /* reserved for kernels that wait inside the device; no present kernel sets it
+                               (disc_project_step reports a wait that ran out through
+                               disc_project_error instead)                                        */
 
 typedef struct disc_set disc_set_t; /* opaque; owns its device memory */
 
@@ -233,6 +237,46 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
               int32_t* node, int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done,
               int32_t* token_out, int32_t* seq_tokens, int32_t seq_ld, float* logq_out,
               float* logp_out, uint32_t* mask_out, uint8_t* status_out, void* stream);
+
+/* One decoding step with the language model's last projection fused in (Algorithm 1, lines 5-8,
+ * where line 5's next-token distribution is softmax(h W / T) of the model's final hidden vectors).
+ *   logit[i][v] = bf16( sum_k hidden[i][k] * wt[v][k] )       (fp32 accumulation, rounded once to
+ * bf16: the value a separate projection would have stored), then exactly disc_step on those logits.
+ * The projection runs on the tensor cores; per row it keeps the sums the log-sum-exp over the
+ * whole vocabulary needs, and writes logits only for the 256-wide vocabulary tiles that hold a
+ * valid next token of the row (all tiles for a row at the empty prefix or at a node with more than
+ * 1024 children), so that for the typical row deep in the prefix tree 512 bytes instead of 2V reach
+ * memory.
+ *   hidden      device, bf16[n][hidden_ld], d values used per row
+ *   wt          device, bf16[V][wt_ld], d values used per row: the vocabulary projection, one
+ *               vocabulary entry per row
+ *   d           model width; a multiple of 8.  hidden, wt, logits_buf and scratch must be 16-byte
+ *               aligned and the row pitches multiples of 16 bytes (DISC_ERR_ARG /
+ *               DISC_ERR_UNSUPPORTED otherwise)
+ *   inv_temperature, seed, step, row_base, state arrays, token_out, seq_tokens, seq_ld, logq_out,
+ *   logp_out, status_out      as for disc_step
+ *   logits_buf  device, bf16[n][logits_ld], logits_ld >= V: receives the logits pieces; with
+ *               store_all != 0 every logit is written (the complete matrix a separate projection
+ *               would have produced: for tests and diagnostics), otherwise what is not written
+ *               keeps its old contents
+ *   scratch     device, disc_project_scratch_bytes(s, n) bytes, caller-owned; its first word is an
+ *               error flag the call clears and the kernel sets when one of its bounded waits ran
+ *               out (read it with disc_project_error)
+ * Rows with NaN or +-Inf logits get DISC_ROW_NONFINITE / DISC_ROW_NOMASS as in disc_step; their
+ * log-weights are not finite but need not equal disc_step's bit for bit.
+ * Three kernels are enqueued on `stream` (tile flags, projection, step); nothing is allocated. */
+int64_t disc_project_scratch_bytes(const disc_set_t* s, int64_t n);
+int disc_project_step(const disc_set_t* s, const void* hidden, int64_t hidden_ld, const void* wt, int64_t wt_ld,
+                      int32_t d, int64_t n, float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base,
+                      int32_t* node, int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done,
+                      int32_t* token_out, int32_t* seq_tokens, int32_t seq_ld, float* logq_out, float* logp_out,
+                      uint8_t* status_out, void* logits_buf, int64_t logits_ld, int32_t store_all, void* scratch,
+                      int64_t scratch_bytes, void* stream);
+
+/* Synchronises `stream` and returns DISC_ERR_CUDA when the projection kernel of an earlier
+ * disc_project_step with this scratch buffer gave up on one of its waits (its results are then
+ * invalid), DISC_OK otherwise. */
+int disc_project_error(const void* scratch, void* stream);
 
 /* K-way importance draw (Algorithm 1, line 22; Appendix A).
  *   logw        device, float[B][K]: log importance scores of the K candidates of each query

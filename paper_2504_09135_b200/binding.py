@@ -24,7 +24,8 @@ ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "D
           -5: "DISC_ERR_OOM", -6: "DISC_ERR_CUDA", -7: "DISC_ERR_UNSUPPORTED"}
 
 EXPORTS = ["disc_build_set", "disc_build_set_eok", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
-           "disc_mask", "disc_mask_static", "disc_verify", "disc_step", "disc_resample", "disc_accept", "disc_accept_resample",
+           "disc_mask", "disc_mask_static", "disc_verify", "disc_step", "disc_project_step", "disc_project_scratch_bytes",
+           "disc_project_error", "disc_resample", "disc_accept", "disc_accept_resample",
            "disc_sampling_uniforms",
            "disc_error_string", "disc_last_cuda_error"]
 
@@ -69,6 +70,10 @@ def lib():
     L.disc_verify.argtypes = [vp, vp, i32, vp, i64, vp, i32, vp, vp, vp, vp, vp, vp]
     L.disc_step.argtypes = [vp, vp, C.c_int, i64, i64, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
                             vp, vp, i32, vp, vp, vp, vp, vp]
+    L.disc_project_step.argtypes = [vp, vp, i64, vp, i64, i32, i64, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
+                                    vp, vp, i32, vp, vp, vp, vp, i64, i32, vp, i64, vp]
+    L.disc_project_scratch_bytes.argtypes = [vp, i64]
+    L.disc_project_error.argtypes = [vp, vp]
     L.disc_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, i32, vp, vp, vp]
     L.disc_accept.argtypes = [vp, i32, i32, u64, i64, vp, vp]
     L.disc_accept_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, vp, i32, vp, vp, vp]
@@ -77,7 +82,9 @@ def lib():
     L.disc_error_string.restype = C.c_char_p
     L.disc_last_cuda_error.argtypes = []
     for name in EXPORTS:
-        if name not in ("disc_free_set", "disc_error_string"):
+        if name == "disc_project_scratch_bytes":
+            getattr(L, name).restype = C.c_int64
+        elif name not in ("disc_free_set", "disc_error_string"):
             getattr(L, name).restype = C.c_int
     _lib = L
     return L
@@ -332,6 +339,50 @@ def disc_step(s: DiscSet, logits: torch.Tensor, state: DiscState, *, inv_tempera
                          _stream_ptr(stream))
     _check(rc, "disc_step")
     return out
+
+
+def disc_project_scratch(s: DiscSet, n: int, device) -> torch.Tensor:
+    """Scratch buffer disc_project_step needs for n rows (caller-owned device memory)."""
+    nbytes = lib().disc_project_scratch_bytes(s.handle, int(n))
+    if nbytes < 0:
+        raise DiscError(int(nbytes), "disc_project_scratch_bytes")
+    return torch.empty(int(nbytes), dtype=torch.uint8, device=device)
+
+
+def disc_project_step(s: DiscSet, hidden: torch.Tensor, wt: torch.Tensor, state: DiscState, logits_buf: torch.Tensor,
+                      scratch: torch.Tensor, *, inv_temperature=1.0, seed=0, step=0, row_base=0,
+                      seq_tokens: torch.Tensor | None = None, out: StepOutputs | None = None, store_all=False,
+                      stream=None) -> StepOutputs:
+    """One step with the last projection fused in: hidden bf16[n, d], wt bf16[V, d] (one vocabulary entry
+    per row), logits_buf bf16[n, >=V] (receives the pieces of the logits the step reads; everything
+    with store_all), scratch from disc_project_scratch."""
+    n = state.n
+    for name, t in (("hidden", hidden), ("wt", wt), ("logits_buf", logits_buf)):
+        if not (t.is_cuda and t.dtype == torch.bfloat16 and t.ndim == 2 and t.stride(1) == 1):
+            raise TypeError(f"{name}: expected a CUDA bfloat16 matrix with unit inner stride")
+    if hidden.shape[0] != n or wt.shape[1] != hidden.shape[1] or logits_buf.shape[0] != n:
+        raise TypeError("disc_project_step: shapes do not fit")
+    if out is None:
+        out = StepOutputs.empty(n, state.node.device)
+    seq_ld = 0 if seq_tokens is None else seq_tokens.shape[-1]
+    rc = lib().disc_project_step(s.handle, hidden.data_ptr(), hidden.stride(0), wt.data_ptr(), wt.stride(0),
+                                 hidden.shape[1], n, float(inv_temperature), int(seed), int(step), int(row_base),
+                                 _dev(state.node, torch.int32, "node"), _dev(state.lo, torch.int32, "lo"),
+                                 _dev(state.hi, torch.int32, "hi"), _dev(state.depth, torch.int32, "depth"),
+                                 _dev(state.logw, torch.float32, "logw"), _dev(state.done, torch.uint8, "done"),
+                                 _dev(out.token, torch.int32, "token"), _dev(seq_tokens, torch.int32, "seq_tokens"),
+                                 seq_ld, _dev(out.logq, torch.float32, "logq"), _dev(out.logp, torch.float32, "logp"),
+                                 _dev(out.status, torch.uint8, "status"), logits_buf.data_ptr(),
+                                 logits_buf.stride(0) if n > 1 else max(logits_buf.shape[1], logits_buf.stride(0)),
+                                 1 if store_all else 0, _dev(scratch, torch.uint8, "scratch"), scratch.numel(),
+                                 _stream_ptr(stream))
+    _check(rc, "disc_project_step")
+    return out
+
+
+def disc_project_check(scratch: torch.Tensor, stream=None) -> None:
+    """Synchronises the stream and raises if the projection kernel gave up on one of its waits."""
+    _check(lib().disc_project_error(_dev(scratch, torch.uint8, "scratch"), _stream_ptr(stream)), "disc_project_error")
 
 
 def disc_resample(logw: torch.Tensor, *, seed=0, query_base=0, seq_tokens: torch.Tensor | None = None,

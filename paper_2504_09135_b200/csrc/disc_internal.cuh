@@ -140,6 +140,13 @@ __device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_
     return make_uint4(c0, c1, c2, c3);
 }
 
+// disc_step with the sums over the whole vocabulary given as per-part (m, s) pairs (disc_step.cu)
+int step_with_parts(const disc_set* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n,
+                    float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base, int32_t* node, int32_t* lo,
+                    int32_t* hi, int32_t* depth, float* logw, uint8_t* done, int32_t* token_out, int32_t* seq_tokens,
+                    int32_t seq_ld, float* logq_out, float* logp_out, uint8_t* status_out, const float2* parts,
+                    int32_t n_parts, cudaStream_t st);
+
 // top 23 bits k of a word -> u = (2k+1) * 2^-24, exact in fp32, as is 1-u
 __device__ __forceinline__ float uniform_from_bits(uint32_t r) {
     return float((r >> 9) * 2u + 1u) * 5.9604644775390625e-08f;

@@ -98,6 +98,10 @@ struct StepParams {
     const uint32_t *root_mask, *heavy_masks;
     int32_t V, W, Wp, n_heavy;
     int64_t M;
+    // the sums over the whole vocabulary given from outside (the fused projection): per row n_parts
+    // pairs (m, s), sum over the part = 2^m * s; used by rows that take the gather path
+    const float2* parts;
+    int32_t n_parts;
 };
 
 // value 2^m * s; the empty sum is (m = -inf, s = 0)
@@ -537,7 +541,10 @@ __device__ void stream_groups_scalar(Acc& a, const RowCtx& r, const PhiloxRoundK
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
-template <int DT, bool VEC>
+// PARTS: rows that take the gather path do not stream their logits; their sum over the whole
+// vocabulary comes from p.parts, and only the logits of their valid tokens are read (the rest of
+// the row need not have been written).
+template <int DT, bool VEC, bool PARTS = false>
 __global__ void __launch_bounds__(STEP_THREADS, DISC_MIN_BLOCKS)
 disc_step_kernel(const __grid_constant__ StepParams p) {
     using E = Elem<DT>;
@@ -562,7 +569,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         if (tid == 0) { p.token_out[row] = -1; p.status_out[row] = DISC_ROW_DONE; }
         return;
     }
-    const float x_first_logit = E::load(rowp, 0);
+    const float x_first_logit = PARTS ? 0.f : E::load(rowp, 0);     // with PARTS element 0 may not have been written
     const int n_groups = (p.V + GROUP - 1) / GROUP;       // the last one may be ragged
     const int n_vec_groups = VEC ? p.V / GROUP : 0;       // whole groups are read with 16-byte loads
 
@@ -633,14 +640,23 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     }
 
     // ---- stream the row
-    if (VEC) {
+    const bool use_parts = PARTS && !dense;
+    MS all_parts{-CUDART_INF_F, 0.f};
+    if (use_parts) {
+        const float2* pr = p.parts + size_t(row) * p.n_parts;
+        for (int j = tid; j < p.n_parts; j += STEP_THREADS) {
+            const float2 v = __ldg(pr + j);
+            all_parts = ms_merge(all_parts, MS{v.x, v.y});
+        }
+        if (v_mine >= 0) x_mine = E::load(rowp, v_mine);
+    } else if (VEC) {
         if (dense) stream_dense<DT>(a, r, p.rk, rowp, gmask, n_vec_groups, flag_tab);
         else stream_sparse<DT>(a, r, rowp, n_vec_groups, [&] { if (v_mine >= 0) x_mine = E::load(rowp, v_mine); });
     } else if (v_mine >= 0) {
         x_mine = E::load(rowp, v_mine);
     }
     if (dense) stream_groups_scalar<DT, true>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
-    else stream_groups_scalar<DT, false>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
+    else if (!use_parts) stream_groups_scalar<DT, false>(a, r, p.rk, rowp, p.V, gmask, n_vec_groups, n_groups);
 
     if (!dense) {
         // ---- gather path: the few allowed logits are read directly.  Every thread adds its child to
@@ -707,6 +723,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     }
 
     MS all = a.touched ? MS{a.mref, (a.sa.x + a.sa.y) + (a.sb.x + a.sb.y)} : MS{-CUDART_INF_F, 0.f};
+    if (use_parts) all = all_parts;
     if (dense) ok = a.touched ? MS{a.mref, a.ok2.x + a.ok2.y} : MS{-CUDART_INF_F, 0.f};
     Best best = a.best;
 
@@ -767,6 +784,9 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         // of flushed terms can win (its score trails the best group by more than the largest noise).
         bool trust = fabsf(l2_all) < CUDART_INF_F && fabsf(l2_ok) < CUDART_INF_F;
         if (dense && !(l2_ok >= all.m - MASS_FLOOR_LOG2)) trust = false;
+        // sums given from outside were formed against exact maxima; the row's logits cannot be
+        // re-read in full, so what the sums say stands (a row with NaN or +Inf gets its status bits)
+        if (use_parts) trust = true;
         s_flag = trust ? 0 : 1;
         red_f[4][0] = best.score; red_i[0][0] = best.key; red_i[1][0] = best.child;
     }
@@ -950,14 +970,47 @@ __global__ void k_sampling_uniforms(PhiloxRoundKeys rk, uint32_t step, uint32_t 
     out[i] = uniform_from_bits(pick_word(r, group_word(G)));
 }
 
-template <int DT, bool VEC>
+template <int DT, bool VEC, bool PARTS = false>
 int launch_step(const StepParams& p, int64_t n, cudaStream_t st) {
-    disc_step_kernel<DT, VEC><<<unsigned(n), STEP_THREADS, 0, st>>>(p);
+    disc_step_kernel<DT, VEC, PARTS><<<unsigned(n), STEP_THREADS, 0, st>>>(p);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }
 
+int fill_step_params(StepParams& p, const disc_set_t* s, const void* logits, int64_t ld, float inv_temperature,
+                     uint64_t seed, uint32_t step, int64_t row_base, int32_t* node, int32_t* lo, int32_t* hi,
+                     int32_t* depth, float* logw, uint8_t* done, int32_t* token_out, int32_t* seq_tokens, int32_t seq_ld,
+                     float* logq_out, float* logp_out, uint32_t* mask_out, uint8_t* status_out) {
+    p.logits = logits; p.ld = ld; p.inv_t = inv_temperature; p.c2 = inv_temperature * LOG2E_F;
+    p.rk = philox_round_keys(seed); p.step = step; p.row_base = uint32_t(row_base);
+    p.node = node; p.lo = lo; p.hi = hi; p.depth = depth; p.logw = logw; p.done = done;
+    p.token_out = token_out; p.seq_tokens = seq_tokens; p.seq_ld = seq_ld;
+    p.logq_out = logq_out; p.logp_out = logp_out; p.mask_out = mask_out; p.status_out = status_out;
+    p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
+    p.root_child = s->root_child; p.root_mask = s->root_mask;
+    p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
+    p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.M = s->M;
+    p.parts = nullptr; p.n_parts = 0;
+    return DISC_OK;
+}
+
 }  // namespace
+
+// disc_step for the fused projection (disc_project.cu): bf16 logits with 16-byte aligned rows of
+// which only the pieces holding valid tokens need to have been written, and the sums over the whole
+// vocabulary as per-part (m, s) pairs.  Arguments are checked by the caller.
+int disc::step_with_parts(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n,
+                          float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base, int32_t* node,
+                          int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done, int32_t* token_out,
+                          int32_t* seq_tokens, int32_t seq_ld, float* logq_out, float* logp_out, uint8_t* status_out,
+                          const float2* parts, int32_t n_parts, cudaStream_t st) {
+    if (dtype != DISC_BF16 || !parts || n_parts <= 0) return DISC_ERR_ARG;
+    StepParams p;
+    fill_step_params(p, s, logits, ld, inv_temperature, seed, step, row_base, node, lo, hi, depth, logw, done, token_out,
+                     seq_tokens, seq_ld, logq_out, logp_out, nullptr, status_out);
+    p.parts = parts; p.n_parts = n_parts;
+    return launch_step<DISC_BF16, true, true>(p, n, st);
+}
 
 extern "C" {
 
@@ -989,15 +1042,8 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
     if (row_base + n > (int64_t(1) << 32)) return DISC_ERR_UNSUPPORTED;
 
     StepParams p;
-    p.logits = logits; p.ld = ld; p.inv_t = inv_temperature; p.c2 = inv_temperature * LOG2E_F;
-    p.rk = philox_round_keys(seed); p.step = step; p.row_base = uint32_t(row_base);
-    p.node = node; p.lo = lo; p.hi = hi; p.depth = depth; p.logw = logw; p.done = done;
-    p.token_out = token_out; p.seq_tokens = seq_tokens; p.seq_ld = seq_ld;
-    p.logq_out = logq_out; p.logp_out = logp_out; p.mask_out = mask_out; p.status_out = status_out;
-    p.node_tok = s->node_tok; p.node_lo = s->node_lo; p.child_begin = s->child_begin;
-    p.root_child = s->root_child; p.root_mask = s->root_mask;
-    p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
-    p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.M = s->M;
+    fill_step_params(p, s, logits, ld, inv_temperature, seed, step, row_base, node, lo, hi, depth, logw, done,
+                     token_out, seq_tokens, seq_ld, logq_out, logp_out, mask_out, status_out);
 
     const size_t esize = dtype == DISC_F32 ? 4 : 2;
     // 16-byte loads need 16-byte aligned rows; other layouts take the scalar path
