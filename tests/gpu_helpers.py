@@ -58,12 +58,17 @@ class LockStep:
         self.checked = 0
         self.max_err = 0.0
 
-    def step(self, logits: torch.Tensor, step: int, seed: int, inv_t: float = 1.0, row_base: int = 0):
+    def step(self, logits, step: int, seed: int, inv_t: float = 1.0, row_base: int = 0, run=None):
+        """run: optional callable(state, seq, out) that performs the step on the GPU some other way
+        than disc_step (the fused projection) and returns the logits tensor that step used."""
         rows = self.rows
         before = {k: getattr(self.state, k).cpu().numpy().copy() for k in ("node", "lo", "hi", "depth", "logw", "done")}
         seq_before = self.seq.cpu().numpy()[rows]
-        disc.disc_step(self.S_gpu, logits, self.state, inv_temperature=inv_t, seed=seed, step=step,
-                       row_base=row_base, seq_tokens=self.seq, out=self.out)
+        if run is not None:
+            logits = run(self.state, self.seq, self.out)
+        else:
+            disc.disc_step(self.S_gpu, logits, self.state, inv_temperature=inv_t, seed=seed, step=step,
+                           row_base=row_base, seq_tokens=self.seq, out=self.out)
         torch.cuda.synchronize()
         g_tok = self.out.token.cpu().numpy()
         g_status = self.out.status.cpu().numpy()

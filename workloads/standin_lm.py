@@ -36,6 +36,19 @@ class StandInLM:
             return out
         return z
 
+    @torch.no_grad()
+    def hidden(self, prev: torch.Tensor) -> torch.Tensor:
+        """The final hidden vectors [R, d] of which logits(prev) is the projection."""
+        return self.E.index_select(0, prev.to(self.device, torch.int64))
+
+    @torch.no_grad()
+    def projection_rows(self) -> torch.Tensor:
+        """The projection with one vocabulary entry per row, [V, d] contiguous (the layout a fused
+        projection kernel takes; the same numbers as W)."""
+        if getattr(self, "_wt", None) is None:
+            self._wt = self.W.t().contiguous()
+        return self._wt
+
     def flops_per_row(self) -> int:
         return 2 * self.d * self.V
 
