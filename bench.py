@@ -50,6 +50,7 @@ def parse_args():
                     help="decode only the first P token positions (profiling: bounds the resident logits)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-fused", action="store_true", help="skip the fused projection + step figure")
     ap.add_argument("--cpu-sample-rows", type=int, default=4096)
     return ap.parse_args()
 
@@ -413,6 +414,12 @@ def run_ours(args):
                            "valid_fraction": round(float(vo["valid"].float().mean().item()), 4)})
         mask_stress["verify_top_m"] = verify
 
+    # ---- the projection fused with the step (secondary figure): a free-running decode per variant,
+    # an event pair around every position; the unfused variant is torch's matmul + disc_step
+    fused = None
+    if rank == 0 and w.logits == "bf16" and not args.no_fused:
+        fused = fused_projection(disc, G, lm, ctx, w, dev, L, seed)
+
     # ---- CPU baseline: the oracle as it stands, on a bounded sample, rank 0 at N = 1 only
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -441,6 +448,7 @@ def run_ours(args):
                                   "(source of the roofline's per-launch times)", "clocks": clocks},
                 "deterministic_replay": same_tokens,
                 "lm_projection_ms_per_position": round(lm_ms, 3), "mask_stress": mask_stress,
+                "fused_projection": fused,
                 "set": {"members": G.N, "entries": G.E, "index_nodes": G.n_nodes,
                         "device_mb": round(G.device_bytes / 1e6, 1), "build_s": round(G.build_seconds, 3)},
                 "setup_s": round(time.time() - t_setup, 1)}
@@ -448,6 +456,67 @@ def run_ours(args):
     G.close()
     if use_dist:
         dist.destroy_process_group()
+
+
+def fused_projection(disc, G, lm, ctx, w, dev, L, seed, reps=3):
+    """Per-position device time of (a) torch matmul + disc_step and (b) disc_project_step, each over
+    its own free-running decode of the workload, from the same contexts."""
+    import torch
+    R = w.R
+    wt = lm.projection_rows()
+    scratch = disc.disc_project_scratch(G, R, dev)
+    logits = torch.empty((R, w.V), dtype=torch.bfloat16, device=dev)
+    seq = torch.empty((R, G.l_max), dtype=torch.int32, device=dev)
+    out = disc.StepOutputs.empty(R, dev)
+    peak_tf = None
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            peak_tf = float(json.load(f).get("bf16_tflops", 0)) or None
+
+    def decode(fused_path):
+        ms = np.zeros(L)
+        live = np.zeros(L, dtype=np.int64)
+        state = disc.disc_state_init(G, R, device=dev)
+        seq.fill_(-1)
+        prev = ctx.to(torch.int64).repeat_interleave(w.K)
+        for t in range(L):
+            live[t] = int((state.done == 0).sum().item())
+            h = lm.hidden(prev)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            if fused_path:
+                disc.disc_project_step(G, h, wt, state, logits, scratch, seed=seed, step=t, seq_tokens=seq, out=out)
+            else:
+                torch.matmul(h, lm.W, out=logits)
+                disc.disc_step(G, logits, state, seed=seed, step=t, seq_tokens=seq, out=out)
+            b.record()
+            torch.cuda.synchronize()
+            ms[t] = a.elapsed_time(b)
+            prev = torch.where(out.token >= 0, out.token.to(torch.int64), prev)
+        if fused_path:
+            disc.disc_project_check(scratch)
+        return ms, live
+
+    res = {}
+    for name, fp in (("unfused", False), ("fused", True)):
+        decode(fp)                                           # warm-up
+        runs = [decode(fp) for _ in range(reps)]
+        ms = np.mean([r[0] for r in runs], axis=0)
+        res[name] = {"ms_per_position": [round(float(x), 4) for x in ms], "ms_per_decode": round(float(ms.sum()), 3),
+                     "live_rows": [int(x) for x in runs[0][1]]}
+    flop = 2.0 * R * w.V * lm.d
+    later = res["fused"]["ms_per_position"][1:] or res["fused"]["ms_per_position"]
+    tf = flop / (float(np.mean(later)) * 1e-3) / 1e12
+    res["flop_per_position"] = flop
+    res["fused_tflops_after_position_0"] = round(tf, 1)
+    res["roofline"] = {"bound": "tensor", "kernel": "disc_project_kernel (+ tile flags + step)", "achieved": round(tf, 1),
+                       "peak": peak_tf, "unit": "TFLOP/s", "frac": None if not peak_tf else round(tf / peak_tf, 4),
+                       "peak_kind": "of measured (cuBLAS bf16 burst)" if peak_tf else "unavailable",
+                       "traffic": None}
+    res["note"] = ("each variant decodes on its own (the projections differ in the last bit of a few logits, so the "
+                   "sampled sequences may part); the projection computes every row, complete or not, in both variants")
+    return res
 
 
 # ----------------------------------------------------------------------------- oracle on the host

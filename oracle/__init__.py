@@ -66,6 +66,12 @@ def lib():
                                   vp, i32, vp, vp, vp,
                                   vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
         L.oracle_step.restype = None
+        L.oracle_topm.argtypes = [vp, C.c_int, i64, i64, i32, i32, vp]
+        L.oracle_topm.restype = None
+        L.oracle_step_topm.argtypes = [vp, vp, C.c_int, i64, i64, i32, C.c_float, u64, u32, vp,
+                                       vp, i32, vp, vp, vp,
+                                       vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
+        L.oracle_step_topm.restype = None
         L.oracle_step_plain.argtypes = [vp, vp, C.c_int, i64, i64, C.c_float, u64, u32, vp,
                                         vp, i32, vp, vp,
                                         vp, vp, vp, vp, vp, vp, vp, vp, vp, vp, C.c_int]
@@ -226,6 +232,41 @@ class OracleSet:
                           _p(o["status"]), int(n_threads))
         return o
 
+    def step_topm(self, logits, dtype, M, prefix, depth, done=None, *, inv_temperature=1.0, seed=0, step=0,
+                  row_ids=None, alt_token=None, n_threads=1):
+        """One decoding step in the paper's top-M mode: the M most probable tokens are verified against
+        the sorted array (Algorithm 2) and the token is drawn among the verified ones.  Outputs as for
+        step(), with n_children = the number of verified candidates; a row without any gets status 1."""
+        depth = _c(depth, np.int32).reshape(-1)
+        n = depth.shape[0]
+        logits = np.ascontiguousarray(logits)
+        assert logits.ndim == 2 and logits.shape[0] == n and logits.shape[1] >= self.V
+        assert logits.dtype == (np.float32 if dtype == F32 else np.uint16)
+        prefix = _c(prefix, np.int32)
+        if prefix.ndim == 1:
+            prefix = prefix.reshape(n, -1)
+        if prefix.shape[1] == 0:
+            prefix = np.zeros((n, 1), dtype=np.int32)
+        done = None if done is None else _c(done, np.uint8)
+        row_ids = None if row_ids is None else _c(row_ids, np.int64)
+        alt_token = None if alt_token is None else _c(alt_token, np.int32)
+        o = {
+            "token": np.empty(n, np.int32), "lo": np.empty(n, np.int32), "hi": np.empty(n, np.int32),
+            "done": np.empty(n, np.uint8), "log_mass": np.empty(n), "lse_all": np.empty(n),
+            "lse_ok": np.empty(n), "logq": np.empty(n), "logp": np.empty(n), "best": np.empty(n),
+            "second": np.empty(n), "alt": np.empty(n), "ingroup_gap": np.empty(n),
+            "n_children": np.empty(n, np.int32),
+            "status": np.empty(n, np.uint8),
+        }
+        lib().oracle_step_topm(self._h, _p(logits), int(dtype), logits.shape[1], n, int(M), float(inv_temperature),
+                               int(seed), int(step), _p(row_ids), _p(prefix), prefix.shape[1], _p(depth),
+                               _p(done), _p(alt_token),
+                               _p(o["token"]), _p(o["lo"]), _p(o["hi"]), _p(o["done"]), _p(o["log_mass"]),
+                               _p(o["lse_all"]), _p(o["lse_ok"]), _p(o["logq"]), _p(o["logp"]),
+                               _p(o["best"]), _p(o["second"]), _p(o["alt"]), _p(o["ingroup_gap"]), _p(o["n_children"]),
+                               _p(o["status"]), int(n_threads))
+        return o
+
     def step_plain(self, logits, dtype, prefix, depth, done=None, *, inv_temperature=1.0, seed=0, step=0,
                    row_ids=None, n_threads=1):
         """The same step with the plain sampler: inverse CDF over the allowed tokens in ascending id,
@@ -270,6 +311,16 @@ class OracleSet:
                                         _p(o["logw32"]), _p(o["idx"]), _p(o["logz"]), int(n_threads))
         assert rc == 0
         return o
+
+
+def topm(logits, dtype, V, M):
+    """Algorithm 2, line 3: the M largest logits of every row (lower id first among equals, NaN last),
+    as token ids in ascending order; int32[n, M], -1 padded when M > V."""
+    logits = np.ascontiguousarray(logits)
+    n = logits.shape[0]
+    cand = np.empty((n, int(M)), np.int32)
+    lib().oracle_topm(_p(logits), int(dtype), logits.shape[1], n, int(V), int(M), _p(cand))
+    return cand
 
 
 def resample(logw, seed=0, query_ids=None):

@@ -318,12 +318,16 @@ struct Lse {
 // One decoding step of one row (Algorithm 1, lines 5-8) from the node its prefix reaches.
 // plain = true draws the token with the plain inverse-CDF sampler instead of the two-stage one;
 // nothing else differs.
+// only: when given, the sorted token ids the mask is restricted to (the verified top-M candidates of
+// Algorithm 2); a child whose token is not among them is treated as not allowed.  With no allowed
+// token left the candidate has run into a dead end: status 1, no token, done.
 StepOut step_row(const Trie& T, int32_t node, const void* logits, int dtype, int64_t base,
                  double inv_t, uint64_t seed, uint32_t step, uint32_t row, int32_t alt_token,
-                 bool plain = false) {
+                 bool plain = false, const std::vector<int32_t>* only = nullptr) {
     StepOut o;
     if (node < 0) { o.status = 1; return o; }                 // prefix not in S
     if (T.first_child[node] < 0) { o.status = 8; o.done = 1; o.lo = T.lo[node]; o.hi = T.hi[node]; return o; }
+    auto allowed = [&](int32_t c) { return !only || std::binary_search(only->begin(), only->end(), T.tok[c]); };
 
     Lse all;
     for (int32_t v = 0; v < T.V; ++v) all.add(load_logit(logits, dtype, base + v) * inv_t);
@@ -353,7 +357,10 @@ StepOut step_row(const Trie& T, int32_t node, const void* logits, int dtype, int
         else if (score > second) second = score;
         cur.clear();
     };
+    int32_t first_allowed = -1;
     for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c]) {
+        if (!allowed(c)) continue;
+        if (first_allowed < 0) first_allowed = c;
         ++o.n_children;
         int32_t v = T.tok[c];
         double z = load_logit(logits, dtype, base + v) * inv_t;
@@ -362,21 +369,26 @@ StepOut step_row(const Trie& T, int32_t node, const void* logits, int dtype, int
         cur.push_back({c, v, z});
     }
     close_group();
-    int32_t best_child = T.first_child[node];                  // lowest id unless a group wins
+    if (first_allowed < 0) {                                   // top-M mode: none of the candidates is valid
+        o.status = 1; o.done = 1; o.log_mass = NEG_INF; o.lse_ok = NEG_INF;
+        return o;
+    }
+    int32_t best_child = first_allowed;                        // lowest id unless a group wins
     if (plain) {
         // Algorithm 1, line 7 as a textbook inverse CDF: weights e^{z_v - max} of the allowed
         // tokens in ascending id, the smallest token whose inclusive cumulative weight exceeds
         // u * total.  No groups, one uniform per (row, step).
         double zmax = NEG_INF, total = 0.0;
         for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c])
-            zmax = std::max(zmax, load_logit(logits, dtype, base + T.tok[c]) * inv_t);
+            if (allowed(c)) zmax = std::max(zmax, load_logit(logits, dtype, base + T.tok[c]) * inv_t);
         if (std::isfinite(zmax)) {
             for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c])
-                total += std::exp(load_logit(logits, dtype, base + T.tok[c]) * inv_t - zmax);
+                if (allowed(c)) total += std::exp(load_logit(logits, dtype, base + T.tok[c]) * inv_t - zmax);
             if (std::isfinite(total) && total > 0.0) {
                 const double target = plain_uniform(seed, step, row) * total;
                 double cum = 0.0;
                 for (int32_t c = T.first_child[node]; c >= 0; c = T.next_sibling[c]) {
+                    if (!allowed(c)) continue;
                     cum += std::exp(load_logit(logits, dtype, base + T.tok[c]) * inv_t - zmax);
                     best_child = c;                            // the last allowed token if rounding leaves cum <= target
                     if (cum > target) break;
@@ -543,6 +555,90 @@ void oracle_verify(const void* h, const int32_t* prefix, int32_t prefix_ld, cons
             if (ok && mask) mask[i * W + (t >> 5)] |= 1u << (t & 31);
         }
     }
+}
+
+// Algorithm 2, line 3: the M tokens of highest probability of one row, i.e. of largest logit.
+// Equal logits are common (bf16 has few distinct values): the lower token id comes first; NaN
+// logits come last.  Returned in ascending token id.
+std::vector<int32_t> top_m_row(const void* logits, int dtype, int64_t base, int32_t V, int32_t M) {
+    std::vector<int32_t> idx(V);
+    for (int32_t v = 0; v < V; ++v) idx[v] = v;
+    auto key = [&](int32_t v) { double z = load_logit(logits, dtype, base + v); return std::isnan(z) ? NEG_INF : z; };
+    auto nan_last = [&](int32_t v) { return std::isnan(load_logit(logits, dtype, base + v)) ? 1 : 0; };
+    std::stable_sort(idx.begin(), idx.end(), [&](int32_t a, int32_t b) {
+        if (nan_last(a) != nan_last(b)) return nan_last(a) < nan_last(b);
+        return key(a) > key(b);
+    });
+    idx.resize(std::min(M, V));
+    std::sort(idx.begin(), idx.end());
+    return idx;
+}
+
+// Algorithm 2, lines 4-5 for one candidate: V_m = a + [t] is located in the sorted array by binary
+// search (the smallest row not smaller than V_m); t is valid iff V_m is a prefix of that row.
+bool verify_candidate(const Trie& T, const int32_t* prefix, int32_t len, int32_t t) {
+    const int64_t N = int64_t(T.sorted_off.size()) - 1;
+    if (t < 0 || t >= T.V) return false;
+    std::vector<int32_t> Vm(prefix, prefix + len);
+    Vm.push_back(t);
+    int64_t a = 0, b = N;
+    while (a < b) {
+        const int64_t mid = (a + b) / 2;
+        const bool smaller = std::lexicographical_compare(T.sorted_tokens.begin() + T.sorted_off[mid],
+                                                          T.sorted_tokens.begin() + T.sorted_off[mid + 1],
+                                                          Vm.begin(), Vm.end());
+        if (smaller) a = mid + 1; else b = mid;
+    }
+    if (a >= N) return false;
+    const int64_t r0 = T.sorted_off[a], r1 = T.sorted_off[a + 1];
+    return (r1 - r0) >= int64_t(Vm.size()) && std::equal(Vm.begin(), Vm.end(), T.sorted_tokens.begin() + r0);
+}
+
+// Top-M candidates of n rows (Algorithm 2, line 3), ascending token id per row; cand is [n][M].
+void oracle_topm(const void* logits, int dtype, int64_t ld, int64_t n, int32_t V, int32_t M, int32_t* cand) {
+    for (int64_t i = 0; i < n; ++i) {
+        std::vector<int32_t> c = top_m_row(logits, dtype, i * ld, V, M);
+        for (int32_t m = 0; m < M; ++m) cand[i * M + m] = m < int32_t(c.size()) ? c[m] : -1;
+    }
+}
+
+// One decoding step in the paper's top-M mode (Algorithm 1, lines 5-8 with the mask of Algorithm 2,
+// lines 3-6): the M most probable tokens are the candidates, each is verified against the sorted
+// array, the token is drawn among the verified ones and the importance score is multiplied by their
+// probability mass.  A row none of whose candidates is valid has reached a dead end (it will fail
+// Algorithm 1's test "a in S"): status 1, token -1, done, log_mass = -inf.  Outputs as for
+// oracle_step; n_valid[i] is the number of verified candidates.
+void oracle_step_topm(const void* h, const void* logits, int dtype, int64_t ld, int64_t n, int32_t M,
+                      float inv_temperature, uint64_t seed, uint32_t step, const int64_t* row_ids,
+                      const int32_t* prefix, int32_t prefix_ld, const int32_t* depth, const uint8_t* done,
+                      const int32_t* alt_token,
+                      int32_t* token, int32_t* lo, int32_t* hi, uint8_t* done_out,
+                      double* log_mass, double* lse_all, double* lse_ok, double* logq, double* logp,
+                      double* best_score, double* second_score, double* alt_score, double* ingroup_gap,
+                      int32_t* n_valid, uint8_t* status, int n_threads) {
+    const Trie& T = *static_cast<const Trie*>(h);
+    parallel_rows(n, n_threads, [&](int64_t i) {
+        StepOut o;
+        if (done && done[i]) {
+            o.status = 8; o.done = 1;
+        } else {
+            const int32_t* pre = prefix + i * prefix_ld;
+            int32_t node = T.walk(pre, depth[i]);
+            uint32_t row = uint32_t(row_ids ? row_ids[i] : i);
+            std::vector<int32_t> cand = top_m_row(logits, dtype, i * ld, T.V, M), ok;
+            for (int32_t t : cand) if (verify_candidate(T, pre, depth[i], t)) ok.push_back(t);
+            o = step_row(T, node, logits, dtype, i * ld, double(inv_temperature), seed, step, row,
+                         alt_token ? alt_token[i] : -1, false, &ok);
+        }
+        token[i] = o.token; lo[i] = o.lo; hi[i] = o.hi; done_out[i] = o.done;
+        log_mass[i] = o.log_mass; lse_all[i] = o.lse_all; lse_ok[i] = o.lse_ok;
+        logq[i] = o.logq; logp[i] = o.logp;
+        best_score[i] = o.best; second_score[i] = o.second;
+        if (alt_score) alt_score[i] = o.alt;
+        if (ingroup_gap) ingroup_gap[i] = o.ingroup_gap;
+        if (n_valid) n_valid[i] = o.n_children;
+        status[i] = o.status;
+    });
 }
 
 // One decoding step for n rows.  Row i's prefix is prefix[i*prefix_ld .. +depth[i]); its logits are
