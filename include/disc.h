@@ -9,6 +9,10 @@
  *                    (Section 2.1) of a prefix a.
  *   disc_verify      Algorithm 2, lines 4-6 as stated: M candidate tokens per prefix verified by
  *                    binary search in the sorted array (top-M mode).
+ *   disc_topm        Algorithm 2, line 3: the M most probable tokens of every row.
+ *   disc_step_topm   Algorithm 1, lines 5-8 with the mask of Algorithm 2 as the paper runs it: the
+ *                    top-M tokens are verified against the sorted array and the token is drawn
+ *                    among the verified ones.
  *   disc_step        Algorithm 1, lines 5-8 for a batch of partial sequences: mask, sample from
  *                    P.mask/|P.mask|_1, append, multiply the importance score by |P.mask|_1.
  *   disc_project_step  the same step with line 5's P = L(a, T) folded in: the model's last projection
@@ -237,6 +241,42 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
               int32_t* node, int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done,
               int32_t* token_out, int32_t* seq_tokens, int32_t seq_ld, float* logq_out,
               float* logp_out, uint32_t* mask_out, uint8_t* status_out, void* stream);
+
+/* Algorithm 2, line 3: the M tokens of largest logit of each of n rows (the M most probable ones).
+ * Equal logits are ordered by token id, the lower id first; NaN logits come last.
+ *   logits, dtype, ld   as for disc_step (device memory; rows of vocab_size values)
+ *   done        device, uint8[n] (nullable): rows with done != 0 are skipped (candidates -1)
+ *   cand_out    device, int32[n][M]: the selected token ids in ascending order, -1 padded when
+ *               M > vocab_size
+ *   lse_out     device, float[n][2] (nullable): the pair (m, s) with
+ *               sum_v 2^(logit_v * log2(e) * inv_temperature) = 2^m * s, a by-product of the passes
+ *               over the row (inv_temperature is used for this output only)
+ * Errors: DISC_ERR_ARG, DISC_ERR_UNSUPPORTED (dtype; n >= 2^31). */
+int disc_topm(const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n, int32_t vocab_size, int32_t M,
+              float inv_temperature, const uint8_t* done, int32_t* cand_out, float* lse_out, void* stream);
+
+/* One decoding step in the paper's top-M mode (Algorithm 1, lines 5-8, with mask = PPV_S(P, a) computed
+ * as Algorithm 2 states it: line 3 selects the M most probable tokens, lines 4-5 verify each
+ * a + [t_m] by binary search in the sorted array, line 6 is the mask of the verified ones).  The
+ * token is drawn among the verified candidates by disc_step's two-stage rule, the importance
+ * log-weight grows by the log of their probability mass.  With M = |V| the result is disc_step's.
+ * A row none of whose candidates is valid has reached a dead end: it would fail Algorithm 1's test
+ * "a in S" (line 15), so it ends here with status DISC_ROW_DEAD, token -1, done = 1 and
+ * logw = -inf (the K-way draw then never picks it).
+ *   M           1 <= M <= 1024
+ *   seq_tokens  device, int32[n][seq_ld], required, seq_ld >= l_max: the tokens produced so far
+ *               (the prefix a of every row, which the verification searches for); the new token
+ *               is appended as in disc_step
+ *   cand_out    device, int32[n][M]: receives the candidates (ascending id)
+ *   scratch     device, disc_step_topm_scratch_bytes(n, M) bytes, 8-byte aligned, caller-owned
+ *   other arguments as for disc_step (mask_out receives the mask of the verified candidates)
+ * Four kernels are enqueued on `stream` (selection, prefix ranges and candidate verification, step). */
+int64_t disc_step_topm_scratch_bytes(int64_t n, int32_t M);
+int disc_step_topm(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n, int32_t M,
+                   float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base, int32_t* node, int32_t* lo,
+                   int32_t* hi, int32_t* depth, float* logw, uint8_t* done, int32_t* token_out, int32_t* seq_tokens,
+                   int32_t seq_ld, float* logq_out, float* logp_out, uint32_t* mask_out, uint8_t* status_out,
+                   int32_t* cand_out, void* scratch, int64_t scratch_bytes, void* stream);
 
 /* One decoding step with the language model's last projection fused in (Algorithm 1, lines 5-8,
  * where line 5's next-token distribution is softmax(h W / T) of the model's final hidden vectors).

@@ -25,7 +25,7 @@ ERRORS = {-1: "DISC_ERR_ARG", -2: "DISC_ERR_EMPTY", -3: "DISC_ERR_TOKEN", -4: "D
 
 EXPORTS = ["disc_build_set", "disc_build_set_eok", "disc_free_set", "disc_set_info", "disc_set_rows", "disc_state_init",
            "disc_mask", "disc_mask_static", "disc_verify", "disc_step", "disc_project_step", "disc_project_scratch_bytes",
-           "disc_project_error", "disc_resample", "disc_accept", "disc_accept_resample",
+           "disc_project_error", "disc_topm", "disc_step_topm", "disc_step_topm_scratch_bytes", "disc_resample", "disc_accept", "disc_accept_resample",
            "disc_sampling_uniforms",
            "disc_error_string", "disc_last_cuda_error"]
 
@@ -72,6 +72,10 @@ def lib():
                             vp, vp, i32, vp, vp, vp, vp, vp]
     L.disc_project_step.argtypes = [vp, vp, i64, vp, i64, i32, i64, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
                                     vp, vp, i32, vp, vp, vp, vp, i64, i32, vp, i64, vp]
+    L.disc_topm.argtypes = [vp, C.c_int, i64, i64, i32, i32, f32, vp, vp, vp, vp]
+    L.disc_step_topm_scratch_bytes.argtypes = [i64, i32]
+    L.disc_step_topm.argtypes = [vp, vp, C.c_int, i64, i64, i32, f32, u64, u32, i64, vp, vp, vp, vp, vp, vp,
+                                 vp, vp, i32, vp, vp, vp, vp, vp, vp, i64, vp]
     L.disc_project_scratch_bytes.argtypes = [vp, i64]
     L.disc_project_error.argtypes = [vp, vp]
     L.disc_resample.argtypes = [vp, i32, i32, u64, i64, vp, vp, vp, i32, vp, vp, vp]
@@ -82,7 +86,7 @@ def lib():
     L.disc_error_string.restype = C.c_char_p
     L.disc_last_cuda_error.argtypes = []
     for name in EXPORTS:
-        if name == "disc_project_scratch_bytes":
+        if name in ("disc_project_scratch_bytes", "disc_step_topm_scratch_bytes"):
             getattr(L, name).restype = C.c_int64
         elif name not in ("disc_free_set", "disc_error_string"):
             getattr(L, name).restype = C.c_int
@@ -339,6 +343,63 @@ def disc_step(s: DiscSet, logits: torch.Tensor, state: DiscState, *, inv_tempera
                          _stream_ptr(stream))
     _check(rc, "disc_step")
     return out
+
+
+def _logits_args(logits: torch.Tensor, n: int, where: str):
+    if logits.dtype == torch.float32:
+        dt = DISC_F32
+    elif logits.dtype == torch.bfloat16:
+        dt = DISC_BF16
+    else:
+        raise DiscError(-7, where)
+    if not (logits.is_cuda and logits.ndim == 2 and logits.shape[0] == n and logits.stride(1) == 1):
+        raise TypeError("logits: expected a CUDA tensor [n, >=V] with unit inner stride")
+    return dt, (logits.stride(0) if n > 1 else max(logits.shape[1], logits.stride(0)))
+
+
+def disc_topm(logits: torch.Tensor, V: int, M: int, *, inv_temperature=1.0, done: torch.Tensor | None = None,
+              want_lse=False, stream=None):
+    """The M largest logits of every row as token ids in ascending order: int32[n, M]; with want_lse
+    also float32[n, 2], the pair (m, s) with sum_v 2^(z_v log2e / T) = 2^m * s."""
+    n = logits.shape[0]
+    dt, ld = _logits_args(logits, n, "disc_topm")
+    cand = torch.empty((n, M), dtype=torch.int32, device=logits.device)
+    lse = torch.empty((n, 2), dtype=torch.float32, device=logits.device) if want_lse else None
+    rc = lib().disc_topm(logits.data_ptr(), dt, ld, n, int(V), int(M), float(inv_temperature),
+                         _dev(done, torch.uint8, "done"), cand.data_ptr(), _dev(lse, torch.float32, "lse"),
+                         _stream_ptr(stream))
+    _check(rc, "disc_topm")
+    return (cand, lse) if want_lse else cand
+
+
+def disc_step_topm(s: DiscSet, logits: torch.Tensor, state: DiscState, M: int, seq_tokens: torch.Tensor, *,
+                   inv_temperature=1.0, seed=0, step=0, row_base=0, out: StepOutputs | None = None,
+                   cand: torch.Tensor | None = None, scratch: torch.Tensor | None = None, stream=None):
+    """One step in the paper's top-M mode.  Returns (StepOutputs, cand int32[n, M])."""
+    n = state.n
+    dt, ld = _logits_args(logits, n, "disc_step_topm")
+    dev = state.node.device
+    if out is None:
+        out = StepOutputs.empty(n, dev)
+    if cand is None:
+        cand = torch.empty((n, M), dtype=torch.int32, device=dev)
+    need = lib().disc_step_topm_scratch_bytes(n, int(M))
+    if need < 0:
+        raise DiscError(int(need), "disc_step_topm_scratch_bytes")
+    if scratch is None:
+        scratch = torch.empty(int(need), dtype=torch.uint8, device=dev)
+    rc = lib().disc_step_topm(s.handle, logits.data_ptr(), dt, ld, n, int(M), float(inv_temperature), int(seed),
+                              int(step), int(row_base), _dev(state.node, torch.int32, "node"),
+                              _dev(state.lo, torch.int32, "lo"), _dev(state.hi, torch.int32, "hi"),
+                              _dev(state.depth, torch.int32, "depth"), _dev(state.logw, torch.float32, "logw"),
+                              _dev(state.done, torch.uint8, "done"), _dev(out.token, torch.int32, "token"),
+                              _dev(seq_tokens, torch.int32, "seq_tokens"), seq_tokens.shape[-1],
+                              _dev(out.logq, torch.float32, "logq"), _dev(out.logp, torch.float32, "logp"),
+                              _dev(out.mask, torch.int32, "mask"), _dev(out.status, torch.uint8, "status"),
+                              _dev(cand, torch.int32, "cand"), _dev(scratch, torch.uint8, "scratch"), scratch.numel(),
+                              _stream_ptr(stream))
+    _check(rc, "disc_step_topm")
+    return out, cand
 
 
 def disc_project_scratch(s: DiscSet, n: int, device) -> torch.Tensor:

@@ -20,7 +20,7 @@ OBJ_DIR = os.path.join(PKG, "build")
 LIB = os.path.join(PKG, "libdisc_b200.so")
 STAMP = LIB + ".sha256"
 
-SOURCES = ["disc_build.cu", "disc_mask.cu", "disc_step.cu", "disc_resample.cu", "disc_verify.cu", "disc_project.cu"]
+SOURCES = ["disc_build.cu", "disc_mask.cu", "disc_step.cu", "disc_resample.cu", "disc_verify.cu", "disc_project.cu", "disc_topm.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

@@ -147,6 +147,13 @@ int step_with_parts(const disc_set* s, const void* logits, disc_dtype_t dtype, i
                     int32_t seq_ld, float* logq_out, float* logp_out, uint8_t* status_out, const float2* parts,
                     int32_t n_parts, cudaStream_t st);
 
+// disc_step in top-M mode (disc_step.cu): the valid set is the verified candidates, the sums come from disc_topm
+int step_with_candidates(const disc_set* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n,
+                         float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base, int32_t* node, int32_t* lo,
+                         int32_t* hi, int32_t* depth, float* logw, uint8_t* done, int32_t* token_out, int32_t* seq_tokens,
+                         int32_t seq_ld, float* logq_out, float* logp_out, uint32_t* mask_out, uint8_t* status_out,
+                         const int32_t* cand, const uint8_t* valid, int32_t M, const float2* lse, cudaStream_t st);
+
 // top 23 bits k of a word -> u = (2k+1) * 2^-24, exact in fp32, as is 1-u
 __device__ __forceinline__ float uniform_from_bits(uint32_t r) {
     return float((r >> 9) * 2u + 1u) * 5.9604644775390625e-08f;

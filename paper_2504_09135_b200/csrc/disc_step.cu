@@ -102,6 +102,11 @@ struct StepParams {
     // pairs (m, s), sum over the part = 2^m * s; used by rows that take the gather path
     const float2* parts;
     int32_t n_parts;
+    // top-M mode: the row's candidate tokens (ascending id) and which of them were verified; the
+    // valid set of the row is the verified candidates instead of the node's children
+    const int32_t* cand;
+    const uint8_t* cand_valid;
+    int32_t cand_M;
 };
 
 // value 2^m * s; the empty sum is (m = -inf, s = 0)
@@ -541,12 +546,20 @@ __device__ void stream_groups_scalar(Acc& a, const RowCtx& r, const PhiloxRoundK
 }
 
 // ---- the kernel ---------------------------------------------------------------------------------
-// PARTS: rows that take the gather path do not stream their logits; their sum over the whole
-// vocabulary comes from p.parts, and only the logits of their valid tokens are read (the rest of
-// the row need not have been written).
-template <int DT, bool VEC, bool PARTS = false>
+// MODE 1 (sums given): rows that take the gather path do not stream their logits; their sum over
+// the whole vocabulary comes from p.parts, and only the logits of their valid tokens are read (the
+// rest of the row need not have been written).
+// MODE 2 (top-M): as mode 1, and the valid set of a row is its verified candidates (p.cand,
+// p.cand_valid; at most TOPM_MAX of them) instead of the children of its node; every row takes the
+// gather path; a row without a verified candidate has run into a dead end.
+constexpr int TOPM_MAX = 1024;
+template <int DT, bool VEC, int MODE = 0>
 __global__ void __launch_bounds__(STEP_THREADS, DISC_MIN_BLOCKS)
 disc_step_kernel(const __grid_constant__ StepParams p) {
+    constexpr bool PARTS = MODE >= 1;
+    constexpr bool LIST = MODE == 2;
+    __shared__ int32_t s_list[LIST ? TOPM_MAX : 1];
+    __shared__ int32_t s_count;
     using E = Elem<DT>;
     __shared__ float red_f[6][STEP_WARPS];
     __shared__ int32_t red_i[2][STEP_WARPS];
@@ -575,7 +588,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 
     int32_t cb = 0, ce = 0;
     if (node >= 0 && int64_t(node) < p.M) { cb = __ldg(p.child_begin + node); ce = __ldg(p.child_begin + node + 1); }
-    const int32_t c = ce - cb;
+    int32_t c = ce - cb;
     if (c <= 0) {   // not a prefix of any member, or already a complete member
         if (tid == 0) {
             p.token_out[row] = -1;
@@ -586,13 +599,43 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         return;
     }
 
+    if (LIST) {
+        // the verified candidates, in ascending id, become the row's valid set
+        if (warp == 0) {
+            const int32_t* cd = p.cand + size_t(row) * p.cand_M;
+            const uint8_t* ok = p.cand_valid + size_t(row) * p.cand_M;
+            int32_t cnt = 0;
+            for (int j0 = 0; j0 < p.cand_M; j0 += 32) {
+                const int j = j0 + lane;
+                const int32_t v = j < p.cand_M ? cd[j] : -1;
+                const bool keep = j < p.cand_M && v >= 0 && v < p.V && ok[j] != 0;
+                const uint32_t bal = __ballot_sync(0xffffffffu, keep);
+                if (keep) s_list[cnt + __popc(bal & ((1u << lane) - 1u))] = v;
+                cnt += __popc(bal);
+            }
+            if (lane == 0) s_count = cnt;
+        }
+        __syncthreads();
+        c = s_count;
+        if (c == 0) {   // none of the candidates extends the prefix: Algorithm 1's "a in S" will fail for this row
+            if (tid == 0) {
+                p.token_out[row] = -1;
+                p.status_out[row] = DISC_ROW_DEAD;
+                p.done[row] = 1;
+                p.logw[row] = -CUDART_INF_F;
+            }
+            return;
+        }
+    }
+    auto kid = [&](int32_t i) -> int32_t { return LIST ? s_list[i] : __ldg(p.node_tok + cb + i); };
+
     // dense rows: locate the prebuilt mask row (root, or a heavy node)
     if (VEC && tid >= 32 && tid < 48) {
         const int f = tid - 32;
         flag_tab[f] = make_float4(float(f & 1), float((f >> 1) & 1), float((f >> 2) & 1), float((f >> 3) & 1));
     }
     int32_t hsel = -2;                                    // -2: not dense
-    if (node == 0 || c > DISC_HEAVY_MIN) {                // the same for every thread of the block
+    if (!LIST && (node == 0 || c > DISC_HEAVY_MIN)) {     // the same for every thread of the block
         if (tid == 0) {
             int32_t h = -2;
             if (node == 0) h = -1;                        // -1: the root's row
@@ -621,8 +664,8 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         } else {
             for (int w = tid; w < p.W; w += STEP_THREADS) mo[w] = 0u;
             __syncthreads();
-            for (int i = cb + tid; i < ce; i += STEP_THREADS) {
-                const int32_t t = __ldg(p.node_tok + i);
+            for (int i = tid; i < c; i += STEP_THREADS) {
+                const int32_t t = kid(i);
                 atomicOr(&mo[t >> 5], 1u << (t & 31));
             }
         }
@@ -630,10 +673,10 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
     // Loads of the gather path and of the final cursor update that can be issued now and used
     // after the row has been streamed: this thread's first child; for a row with a single child
     // (a forced step, the common case deep in the tree) the child's index entries as well.
-    const int32_t v_mine = (!dense && tid < c) ? __ldg(p.node_tok + cb + tid) : -1;
+    const int32_t v_mine = (!dense && tid < c) ? kid(tid) : -1;
     float x_mine = 0.f;
     int32_t only_lo = 0, only_cb = 0, only_ce = 0;
-    if (c == 1 && tid == 0) {
+    if (!LIST && c == 1 && tid == 0) {
         only_lo = __ldg(p.node_lo + cb);
         only_cb = __ldg(p.child_begin + cb);
         only_ce = __ldg(p.child_begin + cb + 1);
@@ -667,15 +710,15 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         // The first child of every thread was fetched before the row was streamed and its logit
         // while the row was streamed (see above).
         for (int i = tid; i < c; i += STEP_THREADS) {
-            const int32_t v = i == tid ? v_mine : __ldg(p.node_tok + cb + i);
+            const int32_t v = i == tid ? v_mine : kid(i);
             const float x = i == tid ? x_mine : E::load(rowp, v);
             ms_add(ok, x, p.c2);
             const int32_t G = v >> 3;
             if (c == 1) {           // a forced step: nothing to draw
-                a.best.score = 0.f; a.best.key = v; a.best.child = cb;
+                a.best.score = 0.f; a.best.key = v; a.best.child = LIST ? -1 : cb;
                 break;
             }
-            const bool leader = (i == 0) || ((__ldg(p.node_tok + cb + i - 1) >> 3) != G);
+            const bool leader = (i == 0) || ((kid(i - 1) >> 3) != G);
             if (leader) {
                 float xs[GROUP];
                 xs[0] = x;
@@ -683,7 +726,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
 #pragma unroll
                 for (int k = 1; k < GROUP; ++k) {
                     if (n == k && i + k < c) {
-                        const int32_t v2 = __ldg(p.node_tok + cb + i + k);
+                        const int32_t v2 = kid(i + k);
                         if ((v2 >> 3) == G) { xs[k] = E::load(rowp, v2); n = k + 1; }
                     }
                 }
@@ -715,8 +758,8 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
                         }
                     }
                     a.best.score = score;
-                    a.best.key = __ldg(p.node_tok + cb + i + pick);
-                    a.best.child = cb + i + pick;
+                    a.best.key = kid(i + pick);
+                    a.best.child = LIST ? -1 : cb + i + pick;
                 }
             }
         }
@@ -810,7 +853,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         }
         if (!dense) {
             for (int i = tid; i < c; i += STEP_THREADS) {
-                const float x = E::load(rowp, __ldg(p.node_tok + cb + i));
+                const float x = E::load(rowp, kid(i));
                 if (x != x) nan_ok = 1; else mx_ok = fmaxf(mx_ok, x);
             }
         }
@@ -840,7 +883,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         }
         if (!dense && fin_ok) {
             for (int i = tid; i < c; i += STEP_THREADS)
-                sum_ok += exp2f(fmaf(E::load(rowp, __ldg(p.node_tok + cb + i)), p.c2, -r_ok));
+                sum_ok += exp2f(fmaf(E::load(rowp, kid(i)), p.c2, -r_ok));
         }
         sum_all = block_sum(sum_all, scratch);
         sum_ok = block_sum(sum_ok, scratch);
@@ -874,7 +917,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
         const int32_t key = red_i[0][0];
         int32_t tok = -1, child = -1;
         if (key < 0) {
-            tok = __ldg(p.node_tok + cb); child = cb;                 // no group with a finite score: lowest id
+            tok = kid(0); child = LIST ? -1 : cb;                     // no group with a finite score: lowest id
         } else if (!dense) {
             tok = key; child = red_i[1][0];                           // drawn in the gather loop already
         } else {
@@ -910,7 +953,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
                     if (((bits >> j) & 1u) && cum[j] > target) pick = j;
             }
             if (pick >= 0) tok = Gw * GROUP + pick;
-            else { tok = __ldg(p.node_tok + cb); child = cb; }
+            else { tok = kid(0); child = LIST ? -1 : cb; }
         }
         if (child < 0) {
             child = (node == 0) ? __ldg(p.root_child + tok) : warp_find_child(p.node_tok, cb, ce, tok);
@@ -939,7 +982,7 @@ disc_step_kernel(const __grid_constant__ StepParams p) {
             if (p.logp_out) p.logp_out[row] = logp;
             p.logw[row] += log_mass;
             p.node[row] = child;
-            if (c == 1) {       // fetched before the row was streamed
+            if (c == 1 && !LIST) {       // fetched before the row was streamed
                 p.lo[row] = only_lo;
                 p.hi[row] = hi_old;
                 p.done[row] = only_cb == only_ce ? 1 : 0;
@@ -970,9 +1013,9 @@ __global__ void k_sampling_uniforms(PhiloxRoundKeys rk, uint32_t step, uint32_t 
     out[i] = uniform_from_bits(pick_word(r, group_word(G)));
 }
 
-template <int DT, bool VEC, bool PARTS = false>
+template <int DT, bool VEC, int MODE = 0>
 int launch_step(const StepParams& p, int64_t n, cudaStream_t st) {
-    disc_step_kernel<DT, VEC, PARTS><<<unsigned(n), STEP_THREADS, 0, st>>>(p);
+    disc_step_kernel<DT, VEC, MODE><<<unsigned(n), STEP_THREADS, 0, st>>>(p);
     DISC_CUDA(cudaGetLastError());
     return DISC_OK;
 }
@@ -991,6 +1034,7 @@ int fill_step_params(StepParams& p, const disc_set_t* s, const void* logits, int
     p.heavy_nodes = s->heavy_nodes; p.heavy_masks = s->heavy_masks; p.n_heavy = s->n_heavy;
     p.V = s->V; p.W = s->W; p.Wp = s->Wp; p.M = s->M;
     p.parts = nullptr; p.n_parts = 0;
+    p.cand = nullptr; p.cand_valid = nullptr; p.cand_M = 0;
     return DISC_OK;
 }
 
@@ -1009,7 +1053,28 @@ int disc::step_with_parts(const disc_set_t* s, const void* logits, disc_dtype_t 
     fill_step_params(p, s, logits, ld, inv_temperature, seed, step, row_base, node, lo, hi, depth, logw, done, token_out,
                      seq_tokens, seq_ld, logq_out, logp_out, nullptr, status_out);
     p.parts = parts; p.n_parts = n_parts;
-    return launch_step<DISC_BF16, true, true>(p, n, st);
+    return launch_step<DISC_BF16, true, 1>(p, n, st);
+}
+
+// disc_step in top-M mode: the valid set of row i is the verified candidates among cand[i][0..M)
+// (ascending id), its sum over the whole vocabulary is lse[i] = (m, s).  Arguments are checked by
+// the caller.
+int disc::step_with_candidates(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64_t ld, int64_t n,
+                               float inv_temperature, uint64_t seed, uint32_t step, int64_t row_base, int32_t* node,
+                               int32_t* lo, int32_t* hi, int32_t* depth, float* logw, uint8_t* done,
+                               int32_t* token_out, int32_t* seq_tokens, int32_t seq_ld, float* logq_out,
+                               float* logp_out, uint32_t* mask_out, uint8_t* status_out, const int32_t* cand,
+                               const uint8_t* valid, int32_t M, const float2* lse, cudaStream_t st) {
+    if (!cand || !valid || !lse || M <= 0 || M > TOPM_MAX) return DISC_ERR_ARG;
+    StepParams p;
+    fill_step_params(p, s, logits, ld, inv_temperature, seed, step, row_base, node, lo, hi, depth, logw, done, token_out,
+                     seq_tokens, seq_ld, logq_out, logp_out, mask_out, status_out);
+    p.parts = lse; p.n_parts = 1;
+    p.cand = cand; p.cand_valid = valid; p.cand_M = M;
+    const size_t esize = dtype == DISC_F32 ? 4 : 2;
+    const bool vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
+    if (dtype == DISC_F32) return vec ? launch_step<DISC_F32, true, 2>(p, n, st) : launch_step<DISC_F32, false, 2>(p, n, st);
+    return vec ? launch_step<DISC_BF16, true, 2>(p, n, st) : launch_step<DISC_BF16, false, 2>(p, n, st);
 }
 
 extern "C" {

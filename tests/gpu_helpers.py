@@ -58,9 +58,11 @@ class LockStep:
         self.checked = 0
         self.max_err = 0.0
 
-    def step(self, logits, step: int, seed: int, inv_t: float = 1.0, row_base: int = 0, run=None):
+    def step(self, logits, step: int, seed: int, inv_t: float = 1.0, row_base: int = 0, run=None, oracle_step=None):
         """run: optional callable(state, seq, out) that performs the step on the GPU some other way
-        than disc_step (the fused projection) and returns the logits tensor that step used."""
+        than disc_step (the fused projection, the top-M mode) and returns the logits tensor that
+        step used.  oracle_step: optional callable with S_cpu.step's signature that takes its place
+        (the top-M mode); rows it ends at a dead end (no token) must end the same way on the GPU."""
         rows = self.rows
         before = {k: getattr(self.state, k).cpu().numpy().copy() for k in ("node", "lo", "hi", "depth", "logw", "done")}
         seq_before = self.seq.cpu().numpy()[rows]
@@ -74,12 +76,22 @@ class LockStep:
         g_status = self.out.status.cpu().numpy()
         after = {k: getattr(self.state, k).cpu().numpy() for k in ("node", "lo", "hi", "depth", "logw", "done")}
         host_logits, dt = logits_to_host(logits[torch.as_tensor(rows, device=logits.device)])
-        o = self.S_cpu.step(host_logits, dt, seq_before, before["depth"][rows], before["done"][rows],
-                            inv_temperature=inv_t, seed=seed, step=step, row_ids=rows + row_base,
-                            alt_token=g_tok[rows], n_threads=8)
+        o = (oracle_step or self.S_cpu.step)(host_logits, dt, seq_before, before["depth"][rows], before["done"][rows],
+                                             inv_temperature=inv_t, seed=seed, step=step, row_ids=rows + row_base,
+                                             alt_token=g_tok[rows], n_threads=8)
         live = before["done"][rows] == 0
+        # rows that ran into a dead end (top-M mode): no token, complete, zero weight, cursor untouched
+        stuck = live & (o["token"] < 0)
+        if stuck.any():
+            assert np.all(g_tok[rows][stuck] == -1) and np.all(g_status[rows][stuck] == o["status"][stuck])
+            assert np.all(after["done"][rows][stuck] == 1) and np.all(after["logw"][rows][stuck] == -np.inf)
+            for k in ("node", "lo", "hi", "depth"):
+                assert np.array_equal(after[k][rows][stuck], before[k][rows][stuck]), k
+        self.stuck = getattr(self, "stuck", 0) + int(stuck.sum())
+        full_live = live
+        live = live & ~stuck
         # rows that were already complete: untouched
-        d = ~live
+        d = ~full_live
         assert np.all(g_tok[rows][d] == -1) and np.all(g_status[rows][d] == disc.ROW_DONE)
         for k in ("node", "lo", "hi", "depth", "logw", "done"):
             assert np.array_equal(after[k][rows][d], before[k][rows][d]), k
