@@ -392,26 +392,39 @@ def run_ours(args):
                        "mask_gbs": round(nbytes / (ms * 1e-3) / 1e9, 1),
                        "frac": round(nbytes / (ms * 1e-3) / 1e9 / peak, 4)}
         del out
-        # top-M verification (Algorithm 2 as stated) of B*K prefixes of the same kind, M = 50 and 500
+        # the paper's top-M mode (Algorithm 2 as stated) on the recorded logits of the first two
+        # positions: selection of the M most probable tokens, their verification in the sorted
+        # array, and the whole top-M step, for the M of the paper's ablation
         nv = dec.R
-        vrng = np.random.default_rng(7)
         verify = []
-        for M in (50, 500):
-            cand = torch.as_tensor(vrng.integers(0, w.V, (nv, M)).astype(np.int32), device=dev)
-            vo = disc.disc_verify(G, pre_d[:nv].contiguous(), len_d[:nv].contiguous(), cand)
-            torch.cuda.synchronize()
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            for _ in range(3):
-                disc.disc_verify(G, pre_d[:nv], len_d[:nv], cand, out=vo)
-            a.record()
-            for _ in range(10):
-                disc.disc_verify(G, pre_d[:nv], len_d[:nv], cand, out=vo)
-            b.record()
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / 10
-            verify.append({"prefixes": nv, "M": M, "ms": round(ms, 4),
-                           "candidates_per_s": round(nv * M / (ms * 1e-3), 1),
-                           "valid_fraction": round(float(vo["valid"].float().mean().item()), 4)})
+        for pos in range(min(2, L)):
+            stp = disc.disc_state_init(G, nv, device=dev)
+            seqp = torch.full((nv, G.l_max), -1, dtype=torch.int32, device=dev)
+            for t in range(pos):                     # bring the rows to this position with the exact mask
+                disc.disc_step(G, logits_steps[t], stp, seed=seed, step=t, seq_tokens=seqp)
+            for M in (50, 100, 500, 1000):
+                def t_ms(fn, reps=5):
+                    fn()
+                    torch.cuda.synchronize()
+                    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    a.record()
+                    for _ in range(reps):
+                        fn()
+                    b.record()
+                    torch.cuda.synchronize()
+                    return a.elapsed_time(b) / reps
+                cand = disc.disc_topm(logits_steps[pos], w.V, M)
+                vo = disc.disc_verify(G, seqp, stp.depth, cand)
+                sel_ms = t_ms(lambda: disc.disc_topm(logits_steps[pos], w.V, M))
+                ver_ms = t_ms(lambda: disc.disc_verify(G, seqp, stp.depth, cand, out=vo))
+                outp = disc.StepOutputs.empty(nv, dev)
+                step_ms = t_ms(lambda: disc.disc_step_topm(G, logits_steps[pos], stp.clone(), M, seqp.clone(),
+                                                           seed=seed, step=pos, out=outp))
+                verify.append({"position": pos, "rows": nv, "M": M, "select_ms": round(sel_ms, 4),
+                               "verify_ms": round(ver_ms, 4), "step_topm_ms": round(step_ms, 4),
+                               "candidates_per_s": round(nv * M / (ver_ms * 1e-3), 1),
+                               "valid_fraction": round(float(vo["valid"].float().mean().item()), 4),
+                               "dead_end_rows": int((outp.status == 1).sum().item())})
         mask_stress["verify_top_m"] = verify
 
     # ---- the projection fused with the step (secondary figure): a free-running decode per variant,

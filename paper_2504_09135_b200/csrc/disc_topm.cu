@@ -3,9 +3,10 @@
 // the whole vocabulary as a pair (m, s) with sum_v 2^(z_v log2e / T) = 2^m * s.
 //
 // One block of 256 threads per row.  A logit is mapped to a 32-bit key whose unsigned order is the
-// order of the values (NaN lowest); the key of the M-th largest logit is found eight bits at a time
-// (a 256-bin histogram of the next byte among the keys that match the bytes found so far; bf16 keys
-// have two significant bytes, fp32 keys four).  A last pass writes out, in ascending token id, every
+// order of the values (NaN lowest); the key of the M-th largest logit is found eleven bits at a
+// time (a 2048-bin histogram in shared memory of the next bits among the keys that match the bits
+// found so far - wide enough that logits of one row seldom meet in a bin; bf16 keys take two such
+// passes, fp32 keys three).  A last pass writes out, in ascending token id, every
 // token whose key is larger, and of the tokens whose key is equal the lowest ids until M are
 // filled: equal logits are common in bf16, and the rule "the lower id first" makes the selection
 // unique.  Every pass streams the row again; after the first it comes from L2.
@@ -82,13 +83,18 @@ __device__ __forceinline__ void for_row(const void* rowp, int V, F f) {
     }
 }
 
+constexpr int RADIX_BITS = 11;
+constexpr int BINS = 1 << RADIX_BITS;
+constexpr int BINS_PER_THREAD = BINS / TOPM_THREADS;
+
 template <int DT, bool VEC>
 __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParams p) {
     constexpr int EPV = Row<DT>::EPV;
-    constexpr int PASSES = DT == DISC_BF16 ? 2 : 4;
-    __shared__ unsigned int hist[TOPM_WARPS][256];
+    constexpr int PASSES = DT == DISC_BF16 ? 2 : 3;
+    __shared__ unsigned int hist[BINS];
     __shared__ unsigned int s_prefix, s_remaining;
     __shared__ float s_red[TOPM_WARPS];
+    __shared__ unsigned int s_wsum[TOPM_WARPS];
     __shared__ int s_scan[TOPM_WARPS][2];
     __shared__ int s_flag;
     const int64_t row = blockIdx.x;
@@ -106,9 +112,11 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
     float row_max = -CUDART_INF_F;     // over the values that are not NaN
     float sum = 0.f;
     for (int pass = 0; pass < PASSES; ++pass) {
-        for (int b = tid; b < TOPM_WARPS * 256; b += TOPM_THREADS) (&hist[0][0])[b] = 0u;
+        for (int b = tid; b < BINS; b += TOPM_THREADS) hist[b] = 0u;
         __syncthreads();
-        const int shift = 24 - 8 * pass;
+        // the window of key bits this pass looks at: [shift, shift + width)
+        const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
+        const int width = pass == 2 ? 10 : 11;
         const uint32_t prefix = s_prefix;
         const float ref = (fabsf(row_max) < CUDART_INF_F) ? row_max * p.c2 : 0.f;
         float mx = -CUDART_INF_F;
@@ -116,14 +124,11 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
         for_row<DT, VEC>(rowp, p.V, [&](int, int e0, const float* x) {
 #pragma unroll
             for (int j = 0; j < EPV; ++j) {
-                const bool in = e0 + j < p.V;
-                const uint32_t key = order_key(x[j]);
-                // the bytes above `shift + 8` must match what earlier passes found
-                const bool match = in && (pass == 0 || (key >> (shift + 8)) == (prefix >> (shift + 8)));
-                const uint32_t bin = match ? ((key >> shift) & 255u) : 256u + uint32_t(lane);   // no peers when unmatched
-                const uint32_t peers = __match_any_sync(FULL, bin);
-                if (match && lane == __ffs(peers) - 1) atomicAdd(&hist[warp][bin], unsigned(__popc(peers)));
-                if (in) {
+                if (e0 + j < p.V) {
+                    const uint32_t key = order_key(x[j]);
+                    // the bits above the window must match what earlier passes found
+                    if (pass == 0 || (key >> (shift + width)) == (prefix >> (shift + width)))
+                        atomicAdd(&hist[(key >> shift) & ((1u << width) - 1u)], 1u);
                     if (pass == 0) { if (x[j] != x[j]) nan_seen = 1; else mx = fmaxf(mx, x[j]); }
                     else if (pass == 1) sum += ex2_approx(fmaf(x[j], p.c2, -ref));
                 }
@@ -141,18 +146,35 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
 #pragma unroll
             for (int w2 = 1; w2 < TOPM_WARPS; ++w2) row_max = fmaxf(row_max, s_red[w2]);
         }
-        if (tid == 0) {
-            // from the largest byte down: the bin that holds the `remaining`-th largest key
-            unsigned int rem = s_remaining;
-            int b = 255;
-            for (; b > 0; --b) {
-                unsigned int cnt = 0;
-                for (int w2 = 0; w2 < TOPM_WARPS; ++w2) cnt += hist[w2][b];
-                if (cnt >= rem) break;
-                rem -= cnt;
+        // From the largest bin down: the bin that holds the `remaining`-th largest key.  Thread t
+        // owns the bins [t*8, t*8+8); `above` = keys in the bins of higher threads.
+        {
+            const unsigned int rem = s_remaining;
+            unsigned int mine = 0;
+#pragma unroll
+            for (int b = 0; b < BINS_PER_THREAD; ++b) mine += hist[tid * BINS_PER_THREAD + b];
+            unsigned int incl = mine;                           // suffix sum over the lanes of the warp
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int v = __shfl_down_sync(FULL, incl, o);
+                if (lane + o < 32) incl += v;
             }
-            s_prefix = prefix | (uint32_t(b) << shift);
-            s_remaining = rem;
+            if (lane == 0) s_wsum[warp] = incl;
+            __syncthreads();
+            unsigned int above = incl - mine;
+            for (int w2 = warp + 1; w2 < TOPM_WARPS; ++w2) above += s_wsum[w2];
+            __syncthreads();
+            if (above < rem && above + mine >= rem) {           // exactly one thread
+                unsigned int left = rem - above;
+                int b = BINS_PER_THREAD - 1;
+                for (; b > 0; --b) {
+                    const unsigned int cnt = hist[tid * BINS_PER_THREAD + b];
+                    if (cnt >= left) break;
+                    left -= cnt;
+                }
+                s_prefix = prefix | (uint32_t(tid * BINS_PER_THREAD + b) << shift);
+                s_remaining = left;
+            }
         }
         __syncthreads();
     }
@@ -185,7 +207,7 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
         for (int j = 0; j < EPV; ++j) {
             if (e0 + j < p.V) {
                 uint32_t key = order_key(x[j]);
-                if (DT == DISC_BF16) key &= 0xffff0000u;      // the low half of a bf16 key is the same for every value of a sign
+                if (DT == DISC_BF16) key &= 0xfffffc00u;      // the passes looked at bits 31..10; the rest is constant for bf16
                 if (key > thr) { ++gt; fl_gt |= 1u << j; }
                 else if (key == thr) { ++eq; fl_eq |= 1u << j; }
             }
