@@ -30,10 +30,29 @@ if ROOT not in sys.path:
 
 METRIC = "disc_decode_tokens_per_s"
 UNIT = "tokens/s"
-# DRAM bytes per disc_step launch measured with ncu (dram__bytes_read.sum + dram__bytes_write.sum),
-# as a ratio to the algorithmic bytes of the captured launches (three positions of the large
-# workload: 3.199 GB of DRAM traffic for 3.1532 GB of algorithmic bytes).
-NCU_TRAFFIC_RATIO = 1.014
+
+
+def ncu_traffic_ratio():
+    """DRAM bytes per algorithmic byte of disc_step_kernel from the committed ncu summary
+    (profiles/disc_step_traffic.txt), or None when the kernel's sources have changed since that
+    capture (the figure would describe another kernel)."""
+    import hashlib
+    try:
+        kv = {}
+        with open(os.path.join(ROOT, "profiles", "disc_step_traffic.txt")) as f:
+            for line in f:
+                if ":" in line and not line.startswith("#"):
+                    k, v = line.split(":", 1)
+                    kv[k.strip()] = v.strip()
+        h = hashlib.sha256()
+        for name in kv["kernel_sources"].split():
+            with open(os.path.join(ROOT, "paper_2504_09135_b200", "csrc", name), "rb") as f:
+                h.update(f.read())
+        if h.hexdigest() != kv["kernel_sources_sha256"]:
+            return None
+        return float(kv["dram_bytes_per_algorithmic_byte"])
+    except (OSError, KeyError, ValueError):
+        return None
 
 
 def parse_args():
@@ -315,8 +334,8 @@ def run_ours(args):
                 "frac_of_nominal_8TBs": round(achieved / 8000.0, 4),
                 "alg_bytes_per_launch": int(kern_bytes / args.steps / len(launches)),
                 "avg_launch_ms": round(kern_ms / args.steps / len(launches), 4),
-                "traffic": (None if NCU_TRAFFIC_RATIO is None
-                            else int(NCU_TRAFFIC_RATIO * kern_bytes / args.steps / len(launches))),
+                "traffic": (None if ncu_traffic_ratio() is None
+                            else int(ncu_traffic_ratio() * kern_bytes / args.steps / len(launches))),
                 "per_step": per_step}
 
     # ---- end to end: logits start in pinned host memory, result read back to the host
