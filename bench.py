@@ -542,7 +542,7 @@ def fused_projection(disc, G, lm, ctx, w, dev, L, seed, reps=3):
     tf = flop / (float(np.mean(later)) * 1e-3) / 1e12
     res["flop_per_position"] = flop
     res["fused_tflops_after_position_0"] = round(tf, 1)
-    res["roofline"] = {"bound": "tensor", "kernel": "disc_project_kernel (+ tile flags + step)", "achieved": round(tf, 1),
+    res["roofline"] = {"bound": "tensor", "kernel": "disc_project_pair_kernel (+ tile flags + step)", "achieved": round(tf, 1),
                        "peak": peak_tf, "unit": "TFLOP/s", "frac": None if not peak_tf else round(tf / peak_tf, 4),
                        "peak_kind": "of measured (cuBLAS bf16 burst)" if peak_tf else "unavailable",
                        "traffic": None}
