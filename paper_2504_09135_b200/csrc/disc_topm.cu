@@ -1,16 +1,31 @@
 // disc_topm: the M most probable tokens of every row (Algorithm 2, line 3), i.e. the M largest
-// logits, by an exact radix selection; and, as a by-product of the same passes, the row's sum over
-// the whole vocabulary as a pair (m, s) with sum_v 2^(z_v log2e / T) = 2^m * s.
+// logits, exactly; and, as a by-product of the same pass, the row's sum over the whole vocabulary
+// as a pair (m, s) with sum_v 2^(z_v log2e / T) = 2^m * s.
 //
-// One block of 256 threads per row.  A logit is mapped to a 32-bit key whose unsigned order is the
-// order of the values (NaN lowest); the key of the M-th largest logit is found eleven bits at a
-// time (a 2048-bin histogram in shared memory of the next bits among the keys that match the bits
-// found so far - wide enough that logits of one row seldom meet in a bin; bf16 keys take two such
-// passes, fp32 keys three).  A last pass writes out, in ascending token id, every
-// token whose key is larger, and of the tokens whose key is equal the lowest ids until M are
-// filled: equal logits are common in bf16, and the rule "the lower id first" makes the selection
-// unique.  Every pass streams the row again; after the first it comes from L2.
+// Order of the values: larger first, -0 = +0, NaN below everything; among equal values the lower
+// token id first, which makes the selection unique (equal logits are common in bf16).
+//
+// Two kernels, one block of 256 threads per row in both.
+//
+// M <= 1024 (the sizes the paper uses): ONE pass over the row.  The block keeps the candidates
+// (order key, token id) in shared memory and a threshold: once M candidates are known, a logit can
+// only matter if it beats the M-th largest value seen so far, so after the first few thousand
+// logits almost nothing passes the test (M ln(V/M) insertions are expected for logits in random
+// order).  The row is read in batches of four 16-byte vectors per thread (16 KB in flight per
+// block); a vector is tested as a whole against the threshold (one packed maximum), so the common
+// case costs the log-sum-exp arithmetic plus a handful of instructions per vector.  When the
+// candidates no longer fit, a radix selection (2048-bin histograms in shared memory over the key
+// bits, eleven at a time, then over the token ids among the keys equal to the M-th) over the stored
+// candidates and the batch at hand keeps exactly the M best and raises the threshold.  Batches are
+// taken in ascending token id, so a later logit that only EQUALS the threshold loses the tie and
+// is dropped by the same test.  A sorted row (every logit beats the threshold) still works: it
+// selects once per batch.  At the end the M ids are sorted by a bitonic network and written out.
+//
+// Larger M: the key of the M-th largest logit is found by histogram passes over the whole row
+// (bf16 keys take two, fp32 keys three), and a last pass writes the selection out in ascending id.
+// Every pass streams the row again; after the first it comes from L2.
 
+#include <cuda_bf16.h>
 #include <math_constants.h>
 
 #include "disc_internal.cuh"
@@ -32,9 +47,11 @@ struct TopmParams {
     float2* lse;             // [n] (nullable)
 };
 
+// unsigned order of the keys = order of the values; -0 and +0 share a key, NaN has the lowest
 __device__ __forceinline__ uint32_t order_key(float x) {
     if (x != x) return 0u;
-    const uint32_t b = __float_as_uint(x);
+    uint32_t b = __float_as_uint(x);
+    if (b == 0x80000000u) b = 0u;
     return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
 }
 __device__ __forceinline__ float ex2_approx(float x) {
@@ -87,37 +104,36 @@ constexpr int RADIX_BITS = 11;
 constexpr int BINS = 1 << RADIX_BITS;
 constexpr int BINS_PER_THREAD = BINS / TOPM_THREADS;
 
+// shared memory of the histogram passes
+struct RadixSmem {
+    unsigned int hist[BINS];
+    unsigned int prefix, remaining;
+    float red[TOPM_WARPS];
+    unsigned int wsum[TOPM_WARPS];
+    int scan[TOPM_WARPS][2];
+    int flag;
+};
+
+// The selection of one row by histogram passes over the whole row (any M); called by the whole block.
 template <int DT, bool VEC>
-__global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParams p) {
+__device__ void radix_row(const TopmParams& p, int64_t row, RadixSmem& sm, bool write_lse) {
     constexpr int EPV = Row<DT>::EPV;
     constexpr int PASSES = DT == DISC_BF16 ? 2 : 3;
-    __shared__ unsigned int hist[BINS];
-    __shared__ unsigned int s_prefix, s_remaining;
-    __shared__ float s_red[TOPM_WARPS];
-    __shared__ unsigned int s_wsum[TOPM_WARPS];
-    __shared__ int s_scan[TOPM_WARPS][2];
-    __shared__ int s_flag;
-    const int64_t row = blockIdx.x;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     int32_t* out = p.cand + size_t(row) * p.M;
-    if (p.done && p.done[row]) {
-        for (int m = tid; m < p.M; m += TOPM_THREADS) out[m] = -1;
-        if (p.lse && tid == 0) p.lse[row] = make_float2(-CUDART_INF_F, 0.f);
-        return;
-    }
     const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * (DT == DISC_BF16 ? 2 : 4);
     const int want = min(p.M, p.V);
-    if (tid == 0) { s_prefix = 0u; s_remaining = unsigned(want); s_flag = 0; }
+    if (tid == 0) { sm.prefix = 0u; sm.remaining = unsigned(want); sm.flag = 0; }
 
     float row_max = -CUDART_INF_F;     // over the values that are not NaN
     float sum = 0.f;
     for (int pass = 0; pass < PASSES; ++pass) {
-        for (int b = tid; b < BINS; b += TOPM_THREADS) hist[b] = 0u;
+        for (int b = tid; b < BINS; b += TOPM_THREADS) sm.hist[b] = 0u;
         __syncthreads();
         // the window of key bits this pass looks at: [shift, shift + width)
         const int shift = pass == 0 ? 21 : (pass == 1 ? 10 : 0);
         const int width = pass == 2 ? 10 : 11;
-        const uint32_t prefix = s_prefix;
+        const uint32_t prefix = sm.prefix;
         const float ref = (fabsf(row_max) < CUDART_INF_F) ? row_max * p.c2 : 0.f;
         float mx = -CUDART_INF_F;
         int nan_seen = 0;
@@ -128,7 +144,7 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
                     const uint32_t key = order_key(x[j]);
                     // the bits above the window must match what earlier passes found
                     if (pass == 0 || (key >> (shift + width)) == (prefix >> (shift + width)))
-                        atomicAdd(&hist[(key >> shift) & ((1u << width) - 1u)], 1u);
+                        atomicAdd(&sm.hist[(key >> shift) & ((1u << width) - 1u)], 1u);
                     if (pass == 0) { if (x[j] != x[j]) nan_seen = 1; else mx = fmaxf(mx, x[j]); }
                     else if (pass == 1) sum += ex2_approx(fmaf(x[j], p.c2, -ref));
                 }
@@ -137,59 +153,59 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
         if (pass == 0) {
 #pragma unroll
             for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
-            if (lane == 0) s_red[warp] = mx;
-            if (nan_seen) s_flag = 1;
+            if (lane == 0) sm.red[warp] = mx;
+            if (nan_seen) sm.flag = 1;
         }
         __syncthreads();
         if (pass == 0) {
-            row_max = s_red[0];
+            row_max = sm.red[0];
 #pragma unroll
-            for (int w2 = 1; w2 < TOPM_WARPS; ++w2) row_max = fmaxf(row_max, s_red[w2]);
+            for (int w2 = 1; w2 < TOPM_WARPS; ++w2) row_max = fmaxf(row_max, sm.red[w2]);
         }
         // From the largest bin down: the bin that holds the `remaining`-th largest key.  Thread t
         // owns the bins [t*8, t*8+8); `above` = keys in the bins of higher threads.
         {
-            const unsigned int rem = s_remaining;
+            const unsigned int rem = sm.remaining;
             unsigned int mine = 0;
 #pragma unroll
-            for (int b = 0; b < BINS_PER_THREAD; ++b) mine += hist[tid * BINS_PER_THREAD + b];
+            for (int b = 0; b < BINS_PER_THREAD; ++b) mine += sm.hist[tid * BINS_PER_THREAD + b];
             unsigned int incl = mine;                           // suffix sum over the lanes of the warp
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const unsigned int v = __shfl_down_sync(FULL, incl, o);
                 if (lane + o < 32) incl += v;
             }
-            if (lane == 0) s_wsum[warp] = incl;
+            if (lane == 0) sm.wsum[warp] = incl;
             __syncthreads();
             unsigned int above = incl - mine;
-            for (int w2 = warp + 1; w2 < TOPM_WARPS; ++w2) above += s_wsum[w2];
+            for (int w2 = warp + 1; w2 < TOPM_WARPS; ++w2) above += sm.wsum[w2];
             __syncthreads();
             if (above < rem && above + mine >= rem) {           // exactly one thread
                 unsigned int left = rem - above;
                 int b = BINS_PER_THREAD - 1;
                 for (; b > 0; --b) {
-                    const unsigned int cnt = hist[tid * BINS_PER_THREAD + b];
+                    const unsigned int cnt = sm.hist[tid * BINS_PER_THREAD + b];
                     if (cnt >= left) break;
                     left -= cnt;
                 }
-                s_prefix = prefix | (uint32_t(tid * BINS_PER_THREAD + b) << shift);
-                s_remaining = left;
+                sm.prefix = prefix | (uint32_t(tid * BINS_PER_THREAD + b) << shift);
+                sm.remaining = left;
             }
         }
         __syncthreads();
     }
-    if (p.lse) {
+    if (p.lse && write_lse) {
         // the row's sum over the whole vocabulary, 2^m * s (NaN or +Inf among the logits poison s)
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
         __syncthreads();
-        if (lane == 0) s_red[warp] = sum;
+        if (lane == 0) sm.red[warp] = sum;
         __syncthreads();
         if (tid == 0) {
             float s = 0.f;
-            for (int w2 = 0; w2 < TOPM_WARPS; ++w2) s += s_red[w2];
+            for (int w2 = 0; w2 < TOPM_WARPS; ++w2) s += sm.red[w2];
             const bool fin = fabsf(row_max) < CUDART_INF_F;
-            if (s_flag || row_max == CUDART_INF_F) s = CUDART_NAN_F;
+            if (sm.flag || row_max == CUDART_INF_F) s = CUDART_NAN_F;
             p.lse[row] = make_float2(row_max == -CUDART_INF_F ? -CUDART_INF_F : (fin ? row_max * p.c2 : 0.f),
                                      row_max == -CUDART_INF_F ? 0.f : s);
         }
@@ -197,8 +213,8 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
 
     // ---- write-out in ascending token id: keys above the threshold, then the lowest ids among the
     // keys equal to it until `want` are filled
-    const uint32_t thr = s_prefix;
-    const int take_eq = int(s_remaining);
+    const uint32_t thr = sm.prefix;
+    const int take_eq = int(sm.remaining);
     int gt_total = 0, eq_total = 0;
     for_row<DT, VEC>(rowp, p.V, [&](int, int e0, const float* x) {
         int gt = 0, eq = 0;
@@ -220,13 +236,13 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
             if (lane >= o) { sg += a; se += b; }
         }
         __syncthreads();
-        if (lane == 31) { s_scan[warp][0] = sg; s_scan[warp][1] = se; }
+        if (lane == 31) { sm.scan[warp][0] = sg; sm.scan[warp][1] = se; }
         __syncthreads();
         int bg = gt_total, be = eq_total, tot_g = 0, tot_e = 0;
 #pragma unroll
         for (int w2 = 0; w2 < TOPM_WARPS; ++w2) {
-            if (w2 < warp) { bg += s_scan[w2][0]; be += s_scan[w2][1]; }
-            tot_g += s_scan[w2][0]; tot_e += s_scan[w2][1];
+            if (w2 < warp) { bg += sm.scan[w2][0]; be += sm.scan[w2][1]; }
+            tot_g += sm.scan[w2][0]; tot_e += sm.scan[w2][1];
         }
         int g_before = bg + sg - gt, e_before = be + se - eq;
 #pragma unroll
@@ -241,6 +257,496 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
         eq_total += tot_e;
     });
     for (int m = want + tid; m < p.M; m += TOPM_THREADS) out[m] = -1;
+}
+
+template <int DT, bool VEC>
+__global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParams p) {
+    __shared__ RadixSmem sm;
+    const int64_t row = blockIdx.x;
+    if (p.done && p.done[row]) {
+        int32_t* out = p.cand + size_t(row) * p.M;
+        for (int m = threadIdx.x; m < p.M; m += TOPM_THREADS) out[m] = -1;
+        if (p.lse && threadIdx.x == 0) p.lse[row] = make_float2(-CUDART_INF_F, 0.f);
+        return;
+    }
+    radix_row<DT, VEC>(p, row, sm, true);
+}
+
+// ---- one pass over the row (M <= 1024) ----------------------------------------------------------------
+#ifndef DISC_TOPM_U
+#define DISC_TOPM_U 8
+#endif
+#ifndef DISC_TOPM_BLOCKS
+#define DISC_TOPM_BLOCKS 4
+#endif
+#ifndef DISC_TOPM_CAP
+#define DISC_TOPM_CAP 3072
+#endif
+constexpr int SEL_U = DISC_TOPM_U;       // 16-byte loads a thread keeps in flight
+constexpr int SEL_SAMPLE = 4;            // vectors per thread in the sample (8192 bf16 or 4096 fp32 logits)
+constexpr int SEL_KEEP = 1024;           // largest M this kernel takes
+constexpr int SEL_CAP = DISC_TOPM_CAP;   // candidates shared memory has room for
+constexpr int SEL_HITS = 2 * SEL_KEEP;   // vectors holding a candidate (kept in the histogram's place)
+
+// the value of a key other than NaN's
+__device__ __forceinline__ float key_value(uint32_t k) {
+    return (k & 0x80000000u) ? __uint_as_float(k & 0x7fffffffu) : __uint_as_float(~k);
+}
+
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+// A 16-byte vector of the row held in registers.
+template <int DT>
+struct Lane;
+template <>
+struct Lane<DISC_BF16> {
+    static constexpr int EPV = 8;
+    __device__ static __forceinline__ void unpack(const uint4& v, float* x) {
+        const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+        for (int j = 0; j < 4; ++j) { x[2 * j] = __uint_as_float(w[j] << 16); x[2 * j + 1] = __uint_as_float(w[j] & 0xffff0000u); }
+    }
+    // the largest element (NaN only if all eight are)
+    __device__ static __forceinline__ float vmax(const uint4& v) {
+        const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.x), *reinterpret_cast<const __nv_bfloat162*>(&v.y));
+        const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.z), *reinterpret_cast<const __nv_bfloat162*>(&v.w));
+        const __nv_bfloat162 c = __hmax2(a, b);
+        const uint32_t w = *reinterpret_cast<const uint32_t*>(&c);
+        return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
+    }
+    // elements id0 .. id0+7 read one by one; -inf where the row has ended
+    __device__ static __forceinline__ uint4 gather(const void* rowp, int id0, int V) {
+        uint32_t w[4];
+        const unsigned short* r = static_cast<const unsigned short*>(rowp);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t lo = (id0 + 2 * j < V) ? uint32_t(__ldg(r + id0 + 2 * j)) : 0xFF80u;
+            const uint32_t hi = (id0 + 2 * j + 1 < V) ? uint32_t(__ldg(r + id0 + 2 * j + 1)) : 0xFF80u;
+            w[j] = lo | (hi << 16);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+template <>
+struct Lane<DISC_F32> {
+    static constexpr int EPV = 4;
+    __device__ static __forceinline__ void unpack(const uint4& v, float* x) {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y); x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+    __device__ static __forceinline__ float vmax(const uint4& v) {
+        return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)), fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
+    }
+    __device__ static __forceinline__ uint4 gather(const void* rowp, int id0, int V) {
+        uint32_t w[4];
+        const uint32_t* r = static_cast<const uint32_t*>(rowp);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) w[j] = (id0 + j < V) ? __ldg(r + id0 + j) : 0xFF800000u;
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+};
+
+// The selections inside a block use 256-bin histograms, one bin per thread, over eight key bits at a
+// time: the candidates are a few hundred, and finding the bin then costs one block-wide suffix sum.
+// Of the keys counted in hist (bins of the key bits [shift, shift+8) among the keys that agree with
+// `prefix` above them), the bin that holds the *rem_io-th largest: *prefix_out gets the bin's bits
+// added, *rem_io its rank inside the bin, *ties_out the bin's count.  Called by the whole block;
+// ends with a barrier.
+__device__ __forceinline__ void pick_bin256(const unsigned int* hist, uint32_t prefix, int shift, unsigned int* s_wsum,
+                                            unsigned int* prefix_out, unsigned int* rem_io, unsigned int* ties_out) {
+    static_assert(TOPM_THREADS == 256, "one bin per thread");
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const unsigned int rem = *rem_io;
+    const unsigned int mine = hist[tid];
+    unsigned int incl = mine;                           // suffix sum over the lanes of the warp
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned int v = __shfl_down_sync(FULL, incl, o);
+        if (lane + o < 32) incl += v;
+    }
+    if (lane == 0) s_wsum[warp] = incl;
+    __syncthreads();
+    unsigned int above = incl - mine;
+#pragma unroll
+    for (int w2 = 1; w2 < TOPM_WARPS; ++w2) above += w2 > warp ? s_wsum[w2] : 0u;
+    __syncthreads();
+    if (above < rem && above + mine >= rem) {           // exactly one thread
+        *prefix_out = prefix | (uint32_t(tid) << shift);
+        *rem_io = rem - above;
+        *ties_out = mine;
+    }
+    __syncthreads();
+}
+
+// Control words of a block's selection, in shared memory.
+struct SelCtl {
+    unsigned int count;        // an allocator: vectors that hold a candidate, then candidates
+    unsigned int prefix, remaining, ties, kept;
+    unsigned int n_sample;
+};
+
+// Of the cnt candidates (keys, ids) in shared memory exactly the `want` best stay, stored in front
+// (c.count = want).  `hist` (2048 words) is scratch: histograms first, then the place the kept
+// candidates are collected in.  Called by the whole block with cnt > want; begins and ends with a
+// barrier.  Out of line: it runs once per row.
+__device__ __noinline__ void select_best(uint32_t* keys, int32_t* ids, unsigned int cnt, unsigned int want, int V,
+                                         bool bf16, unsigned int* hist, unsigned int* s_wsum, SelCtl& c) {
+    const int tid = threadIdx.x;
+    // bf16: the keys differ in their upper 16 bits only
+    const uint32_t key_mask = bf16 ? 0xffff0000u : 0xffffffffu;
+    const int low = bf16 ? 16 : 0;
+    __syncthreads();
+    if (tid == 0) { c.prefix = 0u; c.remaining = want; c.kept = 0u; }
+    for (int shift = 24; shift >= low; shift -= 8) {
+        hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = c.prefix;
+        for (unsigned int i = tid; i < cnt; i += TOPM_THREADS) {
+            const uint32_t k = keys[i];
+            if (shift == 24 || (k >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&hist[(k >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        pick_bin256(hist, prefix, shift, s_wsum, &c.prefix, &c.remaining, &c.ties);
+    }
+    const uint32_t thr_key = c.prefix;            // key (its bits under key_mask) of the want-th best
+    const unsigned int left = c.remaining;        // how many of the candidates with that key stay
+    const unsigned int ties = c.ties;             // how many there are
+    int32_t id_thr = 0x7fffffff;                  // those with an id up to this one
+    if (ties > left) {
+        // the left-th lowest id among the tied candidates: the same search over idmask - id
+        const int nb = 32 - __clz(V - 1);         // V >= 2 here; ids fit nb <= 30 bits
+        const uint32_t idmask = (1u << nb) - 1u;
+        __syncthreads();                          // everyone has read the key search's results
+        if (tid == 0) { c.prefix = 0u; c.remaining = left; }
+        for (int top = nb; top > 0;) {
+            const int shift = max(top - 8, 0);    // the window [shift, top), at most eight bits
+            hist[tid] = 0u;
+            __syncthreads();
+            const uint32_t prefix = c.prefix;
+            for (unsigned int i = tid; i < cnt; i += TOPM_THREADS) {
+                if ((keys[i] & key_mask) == thr_key) {
+                    const uint32_t k2 = idmask - uint32_t(ids[i]);
+                    if (top == nb || (k2 >> top) == (prefix >> top)) atomicAdd(&hist[(k2 >> shift) & ((1u << (top - shift)) - 1u)], 1u);
+                }
+            }
+            __syncthreads();
+            pick_bin256(hist, prefix, shift, s_wsum, &c.prefix, &c.remaining, &c.ties);
+            top = shift;
+        }
+        id_thr = int32_t(idmask - c.prefix);
+    }
+    // the kept candidates are collected in the histogram's place (the last barrier of the search has
+    // passed, nobody reads the histogram any more), then moved to the front
+    uint32_t* tk = hist;
+    int32_t* ti = reinterpret_cast<int32_t*>(hist + SEL_KEEP);
+    for (unsigned int i = tid; i < cnt; i += TOPM_THREADS) {
+        const uint32_t k = keys[i], km = k & key_mask;
+        const int32_t id = ids[i];
+        if (km > thr_key || (km == thr_key && id <= id_thr)) {
+            const unsigned int pos = atomicAdd(&c.kept, 1u);
+            if (pos < unsigned(SEL_KEEP)) { tk[pos] = k; ti[pos] = id; }
+        }
+    }
+    __syncthreads();
+    const unsigned int n_kept = min(c.kept, unsigned(SEL_KEEP));      // = want
+    for (unsigned int i = tid; i < n_kept; i += TOPM_THREADS) { keys[i] = tk[i]; ids[i] = ti[i]; }
+    if (tid == 0) c.count = n_kept;
+    __syncthreads();
+}
+
+template <int DT, bool VEC>
+__global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stream_kernel(const TopmParams p) {
+    using L = Lane<DT>;
+    constexpr int EPV = L::EPV;
+    constexpr int ESIZE = DT == DISC_BF16 ? 2 : 4;
+    constexpr int SAMPLE_VECS = SEL_SAMPLE * TOPM_THREADS;      // vectors of the sample
+    __shared__ uint32_t keys[SEL_CAP];
+    __shared__ int32_t ids[SEL_CAP];
+    __shared__ RadixSmem rs;
+    int32_t* hits = reinterpret_cast<int32_t*>(rs.hist);     // free between the sample's passes and the final selection
+    static_assert(SEL_HITS <= BINS, "the list of vectors fits the histogram's place");
+    __shared__ SelCtl ctl;
+    __shared__ float s_red[2][TOPM_WARPS];
+    __shared__ int s_flag;
+    static_assert(BINS >= 2 * SEL_KEEP, "the histogram's place holds the kept candidates");
+
+    const int64_t row = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    int32_t* out = p.cand + size_t(row) * p.M;
+    if (p.done && p.done[row]) {
+        for (int m = tid; m < p.M; m += TOPM_THREADS) out[m] = -1;
+        if (p.lse && tid == 0) p.lse[row] = make_float2(-CUDART_INF_F, 0.f);
+        return;
+    }
+    const char* rowp = static_cast<const char*>(p.logits) + size_t(row) * size_t(p.ld) * ESIZE;
+    const int V = p.V;
+    const unsigned int want = unsigned(min(p.M, V));
+    const int nvec = (V + EPV - 1) / EPV;
+    auto load_vec = [&](int vi) -> uint4 {
+        const int id0 = vi * EPV;
+        if (VEC && id0 + EPV <= V) return ld_stream16(rowp + size_t(id0) * ESIZE);
+        return L::gather(rowp, id0, V);
+    };
+
+    // ---- A. a threshold from a sample.  SAMPLE_VECS vectors spread evenly over the row (the whole
+    // row if it has no more) are read; with f the sampled share of the row, about want*f of the
+    // row's `want` best are among them, and the r-th best of the sample, r = want*f + 3 sqrt(want*f)
+    // + 1, is below the want-th best of the row except once in some hundred rows.  Whether it was
+    // is known at the end (at least `want` logits reached it); if not, the row is done again by the
+    // histogram passes.
+    // the k-th vector of the sample: runs of 16 vectors (256 bytes), the runs spread evenly
+    auto sample_vec = [&](int k) -> int {
+        if (nvec <= SAMPLE_VECS) return k;
+        return int((int64_t(k >> 4) * nvec) / (SAMPLE_VECS >> 4)) + (k & 15);
+    };
+    uint4 sv[SEL_SAMPLE];
+    unsigned int n_mine = 0u;
+#pragma unroll
+    for (int i = 0; i < SEL_SAMPLE; ++i) {
+        const int k = i * TOPM_THREADS + tid;
+        const int vi = sample_vec(k);
+        sv[i] = load_vec(vi < nvec ? vi : nvec);          // past the end: a vector of -inf that is not counted
+        n_mine += vi < nvec ? unsigned(min(EPV, V - vi * EPV)) : 0u;
+    }
+    if (tid == 0) { ctl.count = 0u; ctl.kept = 0u; ctl.n_sample = 0u; ctl.prefix = 0u; }
+    __syncthreads();
+    {
+        const unsigned int wn = __reduce_add_sync(FULL, n_mine);
+        if (lane == 0) atomicAdd(&ctl.n_sample, wn);
+    }
+    __syncthreads();
+    const unsigned int n_sample = ctl.n_sample;
+    unsigned int r = want;
+    if (unsigned(V) > n_sample) {
+        const float mean = float(want) * float(n_sample) / float(V);
+        r = min(n_sample, unsigned(ceilf(mean + 3.f * sqrtf(mean) + 1.f)));
+    }
+    if (tid == 0) ctl.remaining = r;
+    // The r-th largest key of the sample, eight bits at a time.  The -inf that stands for "past the
+    // end of the row" has the lowest key of all numbers and r counts real logits only, so the
+    // fill never matters.  bf16: the two 16-bit keys of a word are formed together, and a NaN
+    // counts as a large value here (the threshold is then too high and the row is done again).
+#pragma unroll 1
+    for (int shift = 24; shift >= (DT == DISC_BF16 ? 16 : 0); shift -= 8) {
+        rs.hist[tid] = 0u;
+        __syncthreads();
+        const uint32_t prefix = ctl.prefix;
+#pragma unroll
+        for (int i = 0; i < SEL_SAMPLE; ++i) {
+            if (DT == DISC_BF16) {
+                const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    const uint32_t neg = (w[j] & 0x80008000u) >> 15;             // 1 in the halves that are negative
+                    const uint32_t k2 = w[j] ^ ((neg * 0xFFFFu) | 0x80008000u);  // ~h there, h ^ 0x8000 elsewhere
+                    const uint32_t ka = k2 & 0xFFFFu, kb = k2 >> 16;
+                    if (shift == 24) {
+                        atomicAdd(&rs.hist[ka >> 8], 1u);
+                        atomicAdd(&rs.hist[kb >> 8], 1u);
+                    } else {
+                        if ((ka >> 8) == (prefix >> 24)) atomicAdd(&rs.hist[ka & 255u], 1u);
+                        if ((kb >> 8) == (prefix >> 24)) atomicAdd(&rs.hist[kb & 255u], 1u);
+                    }
+                }
+            } else {
+                float x[EPV];
+                L::unpack(sv[i], x);
+#pragma unroll
+                for (int j = 0; j < EPV; ++j) {
+                    const uint32_t key = order_key(x[j]);
+                    if (shift == 24 || (key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&rs.hist[(key >> shift) & 255u], 1u);
+                }
+            }
+        }
+        __syncthreads();
+        pick_bin256(rs.hist, prefix, shift, rs.wsum, &ctl.prefix, &ctl.remaining, &ctl.ties);
+    }
+    // a logit is a candidate if it is at least this (a NaN key: no threshold, every logit is one)
+    float thr = -CUDART_INF_F;
+    {
+        uint32_t full = ctl.prefix;
+        if (DT == DISC_BF16 && !(full & 0x80000000u)) full |= 0xffffu;
+        if (ctl.prefix != 0u) thr = key_value(full);
+    }
+
+    // ---- B. one pass over the row: the sum for the log-sum-exp, and the vectors that hold a candidate
+    // (a vector is tested as a whole; what it holds is looked at in C).  No barriers: thread t
+    // takes the vectors t, t+256, ... with SEL_U loads in flight.
+    float mref = 0.f;
+    float2 acc0 = {0.f, 0.f}, acc1 = {0.f, 0.f};
+    bool touched = false;
+    auto consume = [&](const uint4& raw, int vi) {
+        float x[EPV];
+        L::unpack(raw, x);
+        if (!touched) {
+            float mx = x[0];
+#pragma unroll
+            for (int j = 1; j < EPV; ++j) mx = fmaxf(mx, x[j]);
+            const float m = mx * p.c2;
+            mref = (fabsf(m) < CUDART_INF_F) ? m : 0.f;
+            touched = true;
+        }
+        const float2 cc = make_float2(p.c2, p.c2), nm = make_float2(-mref, -mref);
+#pragma unroll
+        for (int j = 0; j < EPV; j += 4) {
+            const float2 y0 = __ffma2_rn(make_float2(x[j], x[j + 1]), cc, nm);
+            const float2 y1 = __ffma2_rn(make_float2(x[j + 2], x[j + 3]), cc, nm);
+            acc0 = __fadd2_rn(acc0, make_float2(ex2_approx(y0.x), ex2_approx(y0.y)));
+            acc1 = __fadd2_rn(acc1, make_float2(ex2_approx(y1.x), ex2_approx(y1.y)));
+        }
+        if (L::vmax(raw) >= thr) {
+            const unsigned int pos = atomicAdd(&ctl.count, 1u);
+            if (pos < unsigned(SEL_HITS)) hits[pos] = vi;
+        }
+    };
+    {
+        int vi = tid;
+        for (; vi + (SEL_U - 1) * TOPM_THREADS < nvec; vi += SEL_U * TOPM_THREADS) {
+            uint4 raw[SEL_U];
+#pragma unroll
+            for (int u = 0; u < SEL_U; ++u) raw[u] = load_vec(vi + u * TOPM_THREADS);
+#pragma unroll
+            for (int u = 0; u < SEL_U; ++u) consume(raw[u], vi + u * TOPM_THREADS);
+        }
+        for (; vi < nvec; vi += TOPM_THREADS) consume(load_vec(vi), vi);
+    }
+
+    // ---- the row's sum over the whole vocabulary
+    if (p.lse) {
+        float m = touched ? mref : -CUDART_INF_F;
+        float s = (acc0.x + acc0.y) + (acc1.x + acc1.y);
+        float mw = m;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) mw = fmaxf(mw, __shfl_xor_sync(FULL, mw, o));
+        s = (m == -CUDART_INF_F) ? 0.f : s * exp2f(m - mw);
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) s += __shfl_xor_sync(FULL, s, o);
+        if (lane == 0) { s_red[0][warp] = mw; s_red[1][warp] = s; }
+        __syncthreads();
+        float mb = s_red[0][0];
+#pragma unroll
+        for (int w2 = 1; w2 < TOPM_WARPS; ++w2) mb = fmaxf(mb, s_red[0][w2]);
+        float sb = 0.f;
+#pragma unroll
+        for (int w2 = 0; w2 < TOPM_WARPS; ++w2)
+            sb += (s_red[0][w2] == -CUDART_INF_F) ? 0.f : s_red[1][w2] * exp2f(s_red[0][w2] - mb);
+        if (sb > 0.f && sb < CUDART_INF_F) {
+            if (tid == 0) p.lse[row] = make_float2(mb, sb);
+        } else {
+            // Nothing finite, NaN or +Inf among the logits, or a sum that overflowed against the
+            // references of the first logits: the plain way, maximum first, then the sum.
+            float mx = -CUDART_INF_F;
+            int nan_seen = 0;
+            for_row<DT, VEC>(rowp, V, [&](int, int e0, const float* x) {
+#pragma unroll
+                for (int j = 0; j < EPV; ++j)
+                    if (e0 + j < V) { if (x[j] != x[j]) nan_seen = 1; else mx = fmaxf(mx, x[j]); }
+            });
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) mx = fmaxf(mx, __shfl_xor_sync(FULL, mx, o));
+            if (tid == 0) s_flag = 0;
+            __syncthreads();
+            if (lane == 0) s_red[0][warp] = mx;
+            if (nan_seen) s_flag = 1;
+            __syncthreads();
+            float row_max = s_red[0][0];
+#pragma unroll
+            for (int w2 = 1; w2 < TOPM_WARPS; ++w2) row_max = fmaxf(row_max, s_red[0][w2]);
+            const bool fin = fabsf(row_max) < CUDART_INF_F;
+            const float ref = fin ? row_max * p.c2 : 0.f;
+            float sum = 0.f;
+            for_row<DT, VEC>(rowp, V, [&](int, int e0, const float* x) {
+#pragma unroll
+                for (int j = 0; j < EPV; ++j)
+                    if (e0 + j < V) sum += ex2_approx(fmaf(x[j], p.c2, -ref));
+            });
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(FULL, sum, o);
+            if (lane == 0) s_red[1][warp] = sum;
+            __syncthreads();
+            if (tid == 0) {
+                float t = 0.f;
+                for (int w2 = 0; w2 < TOPM_WARPS; ++w2) t += s_red[1][w2];
+                if (s_flag || row_max == CUDART_INF_F) t = CUDART_NAN_F;
+                p.lse[row] = make_float2(row_max == -CUDART_INF_F ? -CUDART_INF_F : ref, row_max == -CUDART_INF_F ? 0.f : t);
+            }
+        }
+    }
+
+    // ---- C. the candidates themselves, the `want` best of them, in ascending id
+    __syncthreads();
+    const unsigned int n_hits = ctl.count;
+    __syncthreads();
+    if (tid == 0) ctl.count = 0u;
+    __syncthreads();
+    bool redo = n_hits > unsigned(SEL_HITS);
+    if (!redo) {
+        for (unsigned int h = tid; h < n_hits; h += TOPM_THREADS) {
+            const int vi = hits[h];
+            float x[EPV];
+            L::unpack(load_vec(vi), x);
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) {
+                if (vi * EPV + j < V && x[j] >= thr) {
+                    const unsigned int pos = atomicAdd(&ctl.count, 1u);
+                    if (pos < unsigned(SEL_CAP)) { keys[pos] = order_key(x[j]); ids[pos] = vi * EPV + j; }
+                }
+            }
+        }
+        __syncthreads();
+        const unsigned int cnt = ctl.count;
+        redo = cnt > unsigned(SEL_CAP) || cnt < want;
+        if (!redo) {
+            unsigned int n = cnt;
+            if (cnt > want) {
+                select_best(keys, ids, cnt, want, V, DT == DISC_BF16, rs.hist, rs.wsum, ctl);
+                n = ctl.count;
+            }
+            // the ids in ascending order: few - every thread counts the ids below its own; many - a
+            // bitonic network over the next power of two
+            __syncthreads();
+            int32_t* tids = reinterpret_cast<int32_t*>(rs.hist);
+            if (n <= unsigned(TOPM_THREADS)) {
+                if (unsigned(tid) < n) {
+                    const int32_t mine = ids[tid];
+                    unsigned int below = 0u;
+                    for (unsigned int j = 0; j < n; ++j) below += ids[j] < mine ? 1u : 0u;
+                    tids[below] = mine;
+                }
+                __syncthreads();
+            } else {
+                unsigned int P = 1u;
+                while (P < n) P <<= 1;
+                for (unsigned int i = tid; i < P; i += TOPM_THREADS) tids[i] = i < n ? ids[i] : 0x7fffffff;
+                __syncthreads();
+                for (unsigned int k = 2u; k <= P; k <<= 1) {
+                    for (unsigned int j = k >> 1; j > 0u; j >>= 1) {
+                        for (unsigned int i = tid; i < P; i += TOPM_THREADS) {
+                            const unsigned int l = i ^ j;
+                            if (l > i) {
+                                const int32_t a = tids[i], c = tids[l];
+                                const bool up = (i & k) == 0u;
+                                if ((a > c) == up) { tids[i] = c; tids[l] = a; }
+                            }
+                        }
+                        __syncthreads();
+                    }
+                }
+            }
+            for (int m = tid; m < p.M; m += TOPM_THREADS) out[m] = unsigned(m) < n ? tids[m] : -1;
+        }
+    }
+    if (redo) {
+        // The sample's threshold was too high (fewer than `want` logits reached it), or too low for
+        // the room there is (rows of equal logits, rows without numbers): the histogram passes.
+        __syncthreads();
+        radix_row<DT, VEC>(p, row, rs, false);
+    }
 }
 
 }  // namespace
@@ -260,7 +766,15 @@ extern "C" int disc_topm(const void* logits, disc_dtype_t dtype, int64_t ld, int
     const bool vec = (reinterpret_cast<uintptr_t>(logits) % 16 == 0) && ((size_t(ld) * esize) % 16 == 0);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const unsigned grid = unsigned(n);
-    if (dtype == DISC_F32) {
+    if (min(M, vocab_size) <= SEL_KEEP) {
+        if (dtype == DISC_F32) {
+            if (vec) disc_topm_stream_kernel<DISC_F32, true><<<grid, TOPM_THREADS, 0, st>>>(p);
+            else disc_topm_stream_kernel<DISC_F32, false><<<grid, TOPM_THREADS, 0, st>>>(p);
+        } else {
+            if (vec) disc_topm_stream_kernel<DISC_BF16, true><<<grid, TOPM_THREADS, 0, st>>>(p);
+            else disc_topm_stream_kernel<DISC_BF16, false><<<grid, TOPM_THREADS, 0, st>>>(p);
+        }
+    } else if (dtype == DISC_F32) {
         if (vec) disc_topm_kernel<DISC_F32, true><<<grid, TOPM_THREADS, 0, st>>>(p);
         else disc_topm_kernel<DISC_F32, false><<<grid, TOPM_THREADS, 0, st>>>(p);
     } else {

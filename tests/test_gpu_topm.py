@@ -26,12 +26,17 @@ def test_top_m_selection_is_the_oracles(dtype, V, pad):
     x[3, rng.integers(0, V, max(1, V // 10))] = -np.inf
     x[4, rng.integers(0, V, 3)] = np.inf
     x[5] = -np.abs(x[5]) - 1.0                         # all negative
+    x[8] = np.sort(x[8])                               # ascending: every logit beats all earlier ones
+    x[9] = np.sort(x[9])[::-1]                         # descending
+    x[10] = -np.abs(np.round(x[10], 0))                # zeros of both signs on top, many ties below
+    x[10, ::3] *= -1.0                                 # (-0.0 * -1 = +0.0, ties across the two zeros)
+    x[11] = np.sort(np.round(x[11], 1))                # ascending with runs of equal values
     logits = torch.as_tensor(x).to(dtype).to(DEV)[:, :V] if pad == 0 else torch.as_tensor(x).to(dtype).to(DEV)[:, :V]
     host, dt = logits_to_host(logits)
     host = np.ascontiguousarray(host)
     done = torch.zeros(n, dtype=torch.uint8, device=DEV)
     done[7] = 1
-    for M in (1, 5, 50, 1000, V, V + 3):
+    for M in (1, 5, 50, 1000, 1024, 1025, V, V + 3):
         cand, lse = disc.disc_topm(logits, V, M, inv_temperature=0.7, done=done, want_lse=True)
         torch.cuda.synchronize()
         want = oracle.topm(host, dt, V, M)
@@ -46,9 +51,36 @@ def test_top_m_selection_is_the_oracles(dtype, V, pad):
     m, s = lse.cpu().numpy()[:, 0].astype(np.float64), lse.cpu().numpy()[:, 1].astype(np.float64)
     with np.errstate(divide="ignore", invalid="ignore"):
         got_lse = (m + np.log2(s)) * np.log(2.0)
-    for i in (0, 2, 3, 5, 6, 8):
+    for i in (0, 2, 3, 5, 6, 8, 9, 10, 11):
         assert close(got_lse[i], logsumexp(z[i])).all(), i
     assert not np.isfinite(got_lse[1]) and not np.isfinite(got_lse[4])      # NaN / +Inf rows are not finite
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_top_m_sum_survives_a_low_temperature(dtype):
+    """The one-pass sum is taken against the first logits a thread sees; with 1/T = 60 a row that
+    rises by a few units overflows it, and the plain two-pass sum has to take over."""
+    from scipy.special import logsumexp
+    rng = np.random.default_rng(11)
+    V, n = 50_000, 6
+    x = (rng.standard_normal((n, V)) * 3).astype(np.float32)
+    x[0] = np.sort(x[0])
+    x[1] = np.sort(x[1])[::-1]
+    x[2] = -300.0
+    x[3, :] = -np.inf
+    logits = torch.as_tensor(x).to(dtype).to(DEV)
+    host, dt = logits_to_host(logits)
+    cand, lse = disc.disc_topm(logits, V, 50, inv_temperature=60.0, want_lse=True)
+    torch.cuda.synchronize()
+    assert np.array_equal(cand.cpu().numpy(), oracle.topm(np.ascontiguousarray(host), dt, V, 50))
+    z = (host.astype(np.float64) if dt == oracle.F32 else (host.astype(np.uint32) << 16).view(np.float32).astype(np.float64))
+    z = z * np.float64(np.float32(60.0))
+    m, s = lse.cpu().numpy()[:, 0].astype(np.float64), lse.cpu().numpy()[:, 1].astype(np.float64)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        got = (m + np.log2(s)) * np.log(2.0)
+    for i in (0, 1, 2, 4, 5):
+        assert close(got[i], logsumexp(z[i])).all(), i
+    assert got[3] == -np.inf
 
 
 CASES = [("llm", dict(n_draws=200_000, B=8, K=16, d=64), 50, 1.0),
