@@ -7,19 +7,24 @@
 //
 // Two kernels, one block of 256 threads per row in both.
 //
-// M <= 1024 (the sizes the paper uses): ONE pass over the row.  The block keeps the candidates
-// (order key, token id) in shared memory and a threshold: once M candidates are known, a logit can
-// only matter if it beats the M-th largest value seen so far, so after the first few thousand
-// logits almost nothing passes the test (M ln(V/M) insertions are expected for logits in random
-// order).  The row is read in batches of four 16-byte vectors per thread (16 KB in flight per
-// block); a vector is tested as a whole against the threshold (one packed maximum), so the common
-// case costs the log-sum-exp arithmetic plus a handful of instructions per vector.  When the
-// candidates no longer fit, a radix selection (2048-bin histograms in shared memory over the key
-// bits, eleven at a time, then over the token ids among the keys equal to the M-th) over the stored
-// candidates and the batch at hand keeps exactly the M best and raises the threshold.  Batches are
-// taken in ascending token id, so a later logit that only EQUALS the threshold loses the tie and
-// is dropped by the same test.  A sorted row (every logit beats the threshold) still works: it
-// selects once per batch.  At the end the M ids are sorted by a bitonic network and written out.
+// M <= 1024 (the sizes the paper uses): ONE pass over the row, in three steps.
+//   A. A threshold from a sample.  8,192 logits spread evenly over the row (runs of 256 bytes) are
+//      read; their r-th largest value is found exactly (256-bin histograms in shared memory over
+//      the key bits, eight at a time), where r is chosen so that this value is below the M-th
+//      largest of the whole row except once in about a thousand rows: with f the sampled share,
+//      the sample holds about Mf of the row's M best, and r = Mf + 3 sqrt(Mf) + 1.
+//   B. The row is streamed once with eight 16-byte loads in flight per thread and no barrier.  The
+//      sum for the log-sum-exp is accumulated, and a vector is tested as a whole against the
+//      threshold (one packed maximum); the few vectors that reach it (about r/f logits do:
+//      some 150 for M = 50, 1,400 for M = 1000) are noted in a list in shared memory.
+//   C. The noted vectors are read again, their logits that reach the threshold become the
+//      candidates (order key, token id), the M best of them are selected exactly (the same
+//      histograms, then over the token ids among the keys equal to the M-th), and the M ids are
+//      sorted and written out.
+//   Whether the threshold was low enough is known in C: at least M logits reached it.  If not, or
+//   if the lists overflowed (a row of equal logits, a row without numbers), the row is done again
+//   by the kernel for larger M below, so the result is exact in every case.  The order in which the
+//   row is read plays no part in it.
 //
 // Larger M: the key of the M-th largest logit is found by histogram passes over the whole row
 // (bf16 keys take two, fp32 keys three), and a last pass writes the selection out in ascending id.
@@ -283,10 +288,9 @@ __global__ void __launch_bounds__(TOPM_THREADS) disc_topm_kernel(const TopmParam
 #define DISC_TOPM_CAP 3072
 #endif
 constexpr int SEL_U = DISC_TOPM_U;       // 16-byte loads a thread keeps in flight
-constexpr int SEL_SAMPLE = 4;            // vectors per thread in the sample (8192 bf16 or 4096 fp32 logits)
 constexpr int SEL_KEEP = 1024;           // largest M this kernel takes
 constexpr int SEL_CAP = DISC_TOPM_CAP;   // candidates shared memory has room for
-constexpr int SEL_HITS = 2 * SEL_KEEP;   // vectors holding a candidate (kept in the histogram's place)
+constexpr int SEL_HITS = 3 * SEL_KEEP;   // vectors holding a candidate
 
 // the value of a key other than NaN's
 __device__ __forceinline__ float key_value(uint32_t k) {
@@ -464,12 +468,12 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     using L = Lane<DT>;
     constexpr int EPV = L::EPV;
     constexpr int ESIZE = DT == DISC_BF16 ? 2 : 4;
+    constexpr int SEL_SAMPLE = DT == DISC_BF16 ? 4 : 8;         // vectors per thread in the sample: 8192 logits
     constexpr int SAMPLE_VECS = SEL_SAMPLE * TOPM_THREADS;      // vectors of the sample
     __shared__ uint32_t keys[SEL_CAP];
     __shared__ int32_t ids[SEL_CAP];
+    __shared__ int32_t hits[SEL_HITS];
     __shared__ RadixSmem rs;
-    int32_t* hits = reinterpret_cast<int32_t*>(rs.hist);     // free between the sample's passes and the final selection
-    static_assert(SEL_HITS <= BINS, "the list of vectors fits the histogram's place");
     __shared__ SelCtl ctl;
     __shared__ float s_red[2][TOPM_WARPS];
     __shared__ int s_flag;
@@ -493,12 +497,22 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
         return L::gather(rowp, id0, V);
     };
 
+    // this thread's share of sum_v 2^(x_v c2 - mref), taken in the first attempt
+    float mref = 0.f;
+    float2 acc0 = {0.f, 0.f}, acc1 = {0.f, 0.f};
+    bool touched = false;
+    // Two attempts.  The second, with a threshold far lower in the sample, runs if the first one's
+    // threshold turned out too high; it costs one more pass over the row (which then comes from L2
+    // in part), a fraction of what the histogram passes cost, so that the odd unlucky row does not
+    // hold up its launch.
+    bool finished = false;
+    for (int attempt = 0; attempt < 2 && !finished; ++attempt) {
+    __syncthreads();
     // ---- A. a threshold from a sample.  SAMPLE_VECS vectors spread evenly over the row (the whole
     // row if it has no more) are read; with f the sampled share of the row, about want*f of the
     // row's `want` best are among them, and the r-th best of the sample, r = want*f + 3 sqrt(want*f)
-    // + 1, is below the want-th best of the row except once in some hundred rows.  Whether it was
-    // is known at the end (at least `want` logits reached it); if not, the row is done again by the
-    // histogram passes.
+    // + 1, is below the want-th best of the row except once in about a thousand rows.  Whether it
+    // was is known at the end (at least `want` logits reached it).
     // the k-th vector of the sample: runs of 16 vectors (256 bytes), the runs spread evenly
     auto sample_vec = [&](int k) -> int {
         if (nvec <= SAMPLE_VECS) return k;
@@ -524,8 +538,11 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     unsigned int r = want;
     if (unsigned(V) > n_sample) {
         const float mean = float(want) * float(n_sample) / float(V);
-        r = min(n_sample, unsigned(ceilf(mean + 3.f * sqrtf(mean) + 1.f)));
+        r = unsigned(ceilf(mean + 3.f * sqrtf(mean) + 1.f));
+        if (attempt) r = 2u * r + 8u;
+        r = min(n_sample, r);
     }
+    const bool can_lower = attempt == 0 && r < n_sample;
     if (tid == 0) ctl.remaining = r;
     // The r-th largest key of the sample, eight bits at a time.  The -inf that stands for "past the
     // end of the row" has the lowest key of all numbers and r counts real logits only, so the
@@ -577,10 +594,8 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     // ---- B. one pass over the row: the sum for the log-sum-exp, and the vectors that hold a candidate
     // (a vector is tested as a whole; what it holds is looked at in C).  No barriers: thread t
     // takes the vectors t, t+256, ... with SEL_U loads in flight.
-    float mref = 0.f;
-    float2 acc0 = {0.f, 0.f}, acc1 = {0.f, 0.f};
-    bool touched = false;
     auto consume = [&](const uint4& raw, int vi) {
+        if (attempt == 0) {
         float x[EPV];
         L::unpack(raw, x);
         if (!touched) {
@@ -598,6 +613,7 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
             const float2 y1 = __ffma2_rn(make_float2(x[j + 2], x[j + 3]), cc, nm);
             acc0 = __fadd2_rn(acc0, make_float2(ex2_approx(y0.x), ex2_approx(y0.y)));
             acc1 = __fadd2_rn(acc1, make_float2(ex2_approx(y1.x), ex2_approx(y1.y)));
+        }
         }
         if (L::vmax(raw) >= thr) {
             const unsigned int pos = atomicAdd(&ctl.count, 1u);
@@ -617,7 +633,7 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     }
 
     // ---- the row's sum over the whole vocabulary
-    if (p.lse) {
+    if (p.lse && attempt == 0) {
         float m = touched ? mref : -CUDART_INF_F;
         float s = (acc0.x + acc0.y) + (acc1.x + acc1.y);
         float mw = m;
@@ -684,7 +700,7 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     __syncthreads();
     if (tid == 0) ctl.count = 0u;
     __syncthreads();
-    bool redo = n_hits > unsigned(SEL_HITS);
+    bool redo = n_hits > unsigned(SEL_HITS), too_few = false;
     if (!redo) {
         for (unsigned int h = tid; h < n_hits; h += TOPM_THREADS) {
             const int vi = hits[h];
@@ -701,6 +717,7 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
         __syncthreads();
         const unsigned int cnt = ctl.count;
         redo = cnt > unsigned(SEL_CAP) || cnt < want;
+        too_few = cnt < want;
         if (!redo) {
             unsigned int n = cnt;
             if (cnt > want) {
@@ -741,9 +758,12 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
             for (int m = tid; m < p.M; m += TOPM_THREADS) out[m] = unsigned(m) < n ? tids[m] : -1;
         }
     }
-    if (redo) {
-        // The sample's threshold was too high (fewer than `want` logits reached it), or too low for
-        // the room there is (rows of equal logits, rows without numbers): the histogram passes.
+    finished = !redo;
+    if (redo && !(too_few && can_lower)) break;      // a lower threshold would not help
+    }
+    if (!finished) {
+        // Both thresholds too high, or too low for the room there is (rows of equal logits, rows
+        // without numbers): the histogram passes.
         __syncthreads();
         radix_row<DT, VEC>(p, row, rs, false);
     }

@@ -83,6 +83,38 @@ def test_top_m_sum_survives_a_low_temperature(dtype):
     assert got[3] == -np.inf
 
 
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_top_m_when_the_sample_misleads(dtype):
+    """The one-pass selection takes its threshold from 8,192 logits in evenly spaced runs of 256
+    bytes.  Rows whose largest logits sit exactly there make that threshold too high: with 15 of
+    them there the second, lower threshold has to succeed, with 1,500 there only the histogram
+    passes can."""
+    V, n, M = 128_256, 4, 50
+    epv = 4 if dtype == torch.float32 else 8
+    nvec, runs = V // epv, 8192 // epv // 16
+    sampled = np.concatenate([np.arange((c * nvec) // runs * epv, ((c * nvec) // runs + 16) * epv) for c in range(runs)])
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((n, V)).astype(np.float32)
+    order = np.argsort(-x, axis=1)
+    for i, n_top in enumerate((15, 1500, 0, 40)):
+        # the n_top largest values of the row go to sampled places, swapped with what was there
+        dst = rng.choice(sampled, n_top, replace=False)
+        src = order[i, :n_top]
+        keep = x[i, dst].copy()
+        x[i, dst] = x[i, src]
+        x[i, src] = keep
+    logits = torch.as_tensor(x).to(dtype).to(DEV)
+    host, dt = logits_to_host(logits)
+    for M in (50, 1000):
+        cand, lse = disc.disc_topm(logits, V, M, want_lse=True)
+        torch.cuda.synchronize()
+        assert np.array_equal(cand.cpu().numpy(), oracle.topm(np.ascontiguousarray(host), dt, V, M)), M
+    from scipy.special import logsumexp
+    z = (host.astype(np.float64) if dt == oracle.F32 else (host.astype(np.uint32) << 16).view(np.float32).astype(np.float64))
+    m, sv = lse.cpu().numpy()[:, 0].astype(np.float64), lse.cpu().numpy()[:, 1].astype(np.float64)
+    assert close((m + np.log2(sv)) * np.log(2.0), logsumexp(z, axis=1)).all()
+
+
 CASES = [("llm", dict(n_draws=200_000, B=8, K=16, d=64), 50, 1.0),
          ("llm", dict(n_draws=50_000, B=4, K=8, d=64, V=32_003), 7, 0.8),
          ("large", dict(n_draws=300_000, B=8, K=16, d=64), 100, 1.0),
