@@ -243,7 +243,8 @@ int disc_step(const disc_set_t* s, const void* logits, disc_dtype_t dtype, int64
               float* logp_out, uint32_t* mask_out, uint8_t* status_out, void* stream);
 
 /* Algorithm 2, line 3: the M tokens of largest logit of each of n rows (the M most probable ones).
- * Equal logits are ordered by token id, the lower id first; NaN logits come last.
+ * Equal logits (-0 and +0 are equal) are ordered by token id, the lower id first; NaN logits come
+ * last.  The selection is exact for every input.
  *   logits, dtype, ld   as for disc_step (device memory; rows of vocab_size values)
  *   done        device, uint8[n] (nullable): rows with done != 0 are skipped (candidates -1)
  *   cand_out    device, int32[n][M]: the selected token ids in ascending order, -1 padded when
