@@ -115,6 +115,38 @@ def test_top_m_when_the_sample_misleads(dtype):
     assert close((m + np.log2(sv)) * np.log(2.0), logsumexp(z, axis=1)).all()
 
 
+def test_top_m_selection_fuzz():
+    """Random shapes, alignments, value distributions and M against the oracle's ordering."""
+    rng = np.random.default_rng(2024)
+    for case in range(48):
+        V = int(rng.choice([1, 2, 7, 8, 9, 255, 256, 257, 1023, 1024, 1025, 2048, 8191, 8192, 8193, 20_000, 33_333]))
+        if case % 3 == 0:
+            V = int(rng.integers(1, 40_000))
+        n = int(rng.integers(1, 6))
+        pad = int(rng.integers(0, 9))
+        dtype = torch.float32 if rng.random() < 0.5 else torch.bfloat16
+        kind = case % 6
+        x = rng.standard_normal((n, V + pad)).astype(np.float32) * float(rng.choice([0.01, 1.0, 30.0]))
+        if kind == 1:
+            x = np.round(x)                              # few distinct values: long runs of ties
+        elif kind == 2:
+            x = rng.standard_cauchy((n, V + pad)).astype(np.float32)
+        elif kind == 3:
+            x[:] = float(rng.standard_normal())          # one value everywhere
+        elif kind == 4:
+            x[rng.random(x.shape) < 0.05] = np.nan
+            x[rng.random(x.shape) < 0.05] = -np.inf
+        elif kind == 5:
+            x = np.sort(x, axis=1) if rng.random() < 0.5 else -np.sort(-x, axis=1)
+        logits = torch.as_tensor(x).to(dtype).to(DEV)[:, :V]
+        host, dt = logits_to_host(logits)
+        host = np.ascontiguousarray(host)
+        for M in {1, int(rng.integers(1, 1025)), min(V, 1024), int(rng.integers(1, 3000))}:
+            cand = disc.disc_topm(logits, V, M)
+            torch.cuda.synchronize()
+            assert np.array_equal(cand.cpu().numpy(), oracle.topm(host, dt, V, M)), (case, V, pad, dtype, kind, M)
+
+
 CASES = [("llm", dict(n_draws=200_000, B=8, K=16, d=64), 50, 1.0),
          ("llm", dict(n_draws=50_000, B=4, K=8, d=64, V=32_003), 7, 0.8),
          ("large", dict(n_draws=300_000, B=8, K=16, d=64), 100, 1.0),
