@@ -10,9 +10,11 @@
 //      range [lo, hi) of X; both ends come from one binary search each, with the lanes comparing
 //      the positions of a row against a in parallel (first difference decides; a row that ends
 //      inside a is smaller).
-//   2. verify_candidates_kernel, one thread per candidate: inside [lo, hi) all rows agree with a,
-//      so V_m is located by a binary search on the single column |a|.  The search lands on the
-//      same row index as a search over all of X would.
+//   2. inside [lo, hi) all rows agree with a, so V_m is located by a binary search on the single
+//      column |a|; the search lands on the same row index as a search over all of X would.  One
+//      thread per candidate when a prefix has few (verify_candidates_kernel); with 128 or more, one
+//      block per prefix that first narrows every search between two of 256 pivot rows held in
+//      shared memory (verify_candidates_pivot_kernel).
 // Rows are ragged (no padding token): a row shorter than the compared position counts as smaller.
 
 #include "disc_internal.cuh"
@@ -85,28 +87,78 @@ __global__ void __launch_bounds__(VR_THREADS) verify_range_kernel(const VerifyPa
     }
 }
 
+// What the searches of one prefix share: its range, the column, and where the search starts.
+// Inside [lo, hi) every row has the prefix, so it has at least d tokens; only a row that IS the
+// prefix has exactly d, and it sorts first.  It is smaller than every a + [t], so the searches skip
+// it and a row's key is simply its token at column d (two dependent loads per probe, not three).
+struct RowRange {
+    int32_t lo, hi, d, first;     // first: the first row the searches look at (lo or lo + 1)
+};
+__device__ __forceinline__ RowRange row_range(const VerifyParams& p, int64_t i) {
+    RowRange r;
+    r.lo = p.lo_out[i];
+    r.hi = p.hi_out[i];
+    r.d = p.prefix_len[i];
+    if (r.d < 0 || r.d > p.prefix_ld || r.d > DISC_MAX_DEPTH) r.d = 0;      // such a prefix got the empty range
+    r.first = r.lo;
+    if (r.lo < r.hi && int32_t(__ldg(p.row_off + r.lo + 1) - __ldg(p.row_off + r.lo)) <= r.d) r.first = r.lo + 1;
+    return r;
+}
+__device__ __forceinline__ int32_t key_at(const VerifyParams& p, int32_t j, int32_t d) {
+    return __ldg(p.tok + __ldg(p.row_off + j) + d);
+}
+// the first row of [x, y) whose key is not below t (y if there is none), then the verdict
+__device__ __forceinline__ void finish_candidate(const VerifyParams& p, const RowRange& r, int64_t i, int64_t g, int32_t t,
+                                                 int32_t x, int32_t y) {
+    while (x < y) {
+        const int32_t mid = x + ((y - x) >> 1);
+        if (key_at(p, mid, r.d) < t) x = mid + 1; else y = mid;
+    }
+    const bool ok = t >= 0 && t < p.V && x < r.hi && key_at(p, x, r.d) == t;
+    p.valid_out[g] = ok ? 1 : 0;
+    if (p.row_out) p.row_out[g] = x;
+    if (ok && p.mask_out) atomicOr(p.mask_out + i * p.W + (t >> 5), 1u << (t & 31));
+}
+
+// Few candidates per prefix: one thread per candidate.
 __global__ void __launch_bounds__(256) verify_candidates_kernel(const VerifyParams p) {
     const int64_t g = int64_t(blockIdx.x) * blockDim.x + threadIdx.x;
     if (g >= p.n * p.M) return;
     const int64_t i = g / p.M;
-    const int32_t t = p.cand[g];
-    const int32_t lo = p.lo_out[i], hi = p.hi_out[i];
-    int32_t d = p.prefix_len[i];
-    if (d < 0 || d > p.prefix_ld || d > DISC_MAX_DEPTH) d = 0;      // such a prefix got the empty range
-    // token of row j at column d; a row that ends before it is smaller than every candidate
-    auto key = [&](int32_t j) -> int32_t {
-        const uint32_t b = __ldg(p.row_off + j), e = __ldg(p.row_off + j + 1);
-        return (int32_t(e - b) > d) ? __ldg(p.tok + b + d) : INT32_MIN;
-    };
-    int32_t x = lo, y = hi;                          // the first row with key >= t is in [x, y]
-    while (x < y) {
-        const int32_t mid = x + ((y - x) >> 1);
-        if (key(mid) < t) x = mid + 1; else y = mid;
+    const RowRange r = row_range(p, i);
+    finish_candidate(p, r, i, g, p.cand[g], r.first, r.hi);
+}
+
+// Many candidates per prefix: one block per prefix.  The block first reads the keys of VP evenly
+// spaced rows of the range into shared memory; a candidate finds its place among these pivots
+// there (8 steps that touch no global memory) and searches only between two neighbouring pivots.
+// The searches of a prefix all run over the same rows, so the pivots' 2 x VP loads replace eight
+// probes of every candidate.
+constexpr int VP = 256;
+__global__ void __launch_bounds__(VP) verify_candidates_pivot_kernel(const VerifyParams p) {
+    __shared__ int32_t piv[VP];
+    const int64_t i = blockIdx.x;
+    const RowRange r = row_range(p, i);
+    const int64_t span = int64_t(r.hi) - r.first;
+    const bool use_piv = span > 4 * VP;
+    auto pos = [&](int k) -> int32_t { return r.first + int32_t((int64_t(k + 1) * span) / (VP + 1)); };   // k = 0 .. VP-1
+    if (use_piv) piv[threadIdx.x] = key_at(p, pos(threadIdx.x), r.d);
+    __syncthreads();
+    for (int m = threadIdx.x; m < p.M; m += VP) {
+        const int64_t g = i * p.M + m;
+        const int32_t t = p.cand[g];
+        int32_t x = r.first, y = r.hi;
+        if (use_piv) {
+            int a = 0, b = VP;                      // the first pivot whose key is not below t
+            while (a < b) {
+                const int mid = (a + b) >> 1;
+                if (piv[mid] < t) a = mid + 1; else b = mid;
+            }
+            if (a > 0) x = pos(a - 1) + 1;
+            if (a < VP) y = pos(a);
+        }
+        finish_candidate(p, r, i, g, t, x, y);
     }
-    const bool ok = t >= 0 && t < p.V && x < hi && key(x) == t;
-    p.valid_out[g] = ok ? 1 : 0;
-    if (p.row_out) p.row_out[g] = x;
-    if (ok && p.mask_out) atomicOr(p.mask_out + i * p.W + (t >> 5), 1u << (t & 31));
 }
 
 }  // namespace
@@ -130,8 +182,12 @@ extern "C" int disc_verify(const disc_set_t* s, const int32_t* prefix, int32_t p
     verify_range_kernel<<<unsigned((n + VR_WARPS - 1) / VR_WARPS), VR_THREADS, 0, st>>>(p);
     DISC_CUDA(cudaGetLastError());
     if (M > 0) {
-        const int64_t total = n * M;
-        verify_candidates_kernel<<<unsigned((total + 255) / 256), 256, 0, st>>>(p);
+        if (M >= 128) {
+            verify_candidates_pivot_kernel<<<unsigned(n), VP, 0, st>>>(p);
+        } else {
+            const int64_t total = n * M;
+            verify_candidates_kernel<<<unsigned((total + 255) / 256), 256, 0, st>>>(p);
+        }
         DISC_CUDA(cudaGetLastError());
     }
     return DISC_OK;

@@ -333,7 +333,10 @@ def test_accept_then_resample_parity(K):
 
 @pytest.mark.parametrize("name,over,n,M", [("tiny", {}, 300, 9), ("genret", {}, 1500, 50),
                                            ("llm", dict(n_draws=200_000), 1500, 50),
-                                           ("large", dict(n_draws=300_000), 1200, 100)])
+                                           ("large", dict(n_draws=300_000), 1200, 100),
+                                           ("large", dict(n_draws=300_000), 600, 300),      # one block per prefix, pivots
+                                           ("llm", dict(n_draws=200_000), 300, 1000),
+                                           ("tiny", {}, 200, 128)])
 def test_verify_parity(name, over, n, M):
     """disc_verify (Algorithm 2, lines 4-6: binary search in the sorted array) against the oracle:
     validity, the row every search lands on, the extended mask, the prefix's member range."""
