@@ -9,10 +9,12 @@
 //
 // M <= 1024 (the sizes the paper uses): ONE pass over the row, in three steps.
 //   A. A threshold from a sample.  8,192 logits spread evenly over the row (runs of 256 bytes) are
-//      read; their r-th largest value is found exactly (256-bin histograms in shared memory over
-//      the key bits, eight at a time), where r is chosen so that this value is below the M-th
-//      largest of the whole row except once in about a thousand rows: with f the sampled share,
-//      the sample holds about Mf of the row's M best, and r = Mf + 3 sqrt(Mf) + 1.
+//      read, 32 per thread; the r-th largest of the 256 threads' maxima (256-bin histograms in
+//      shared memory over the key bits, eight at a time) is at most the r-th largest of the
+//      sample, and r is chosen so that this is below the M-th largest of the whole row except
+//      once in about a thousand rows: with f the sampled share, the sample holds about Mf of the
+//      row's M best, and r = Mf + 3 sqrt(Mf) + 1.  (A row no longer than the sample is its own
+//      sample, and the M-th largest is found exactly.)
 //   B. The row is streamed once with eight 16-byte loads in flight per thread and no barrier.  The
 //      sum for the log-sum-exp is accumulated, and a vector is tested as a whole against the
 //      threshold (one packed maximum); the few vectors that reach it (about r/f logits do:
@@ -544,44 +546,66 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     }
     const bool can_lower = attempt == 0 && r < n_sample;
     if (tid == 0) ctl.remaining = r;
-    // The r-th largest key of the sample, eight bits at a time.  The -inf that stands for "past the
-    // end of the row" has the lowest key of all numbers and r counts real logits only, so the
-    // fill never matters.  bf16: the two 16-bit keys of a word are formed together, and a NaN
-    // counts as a large value here (the threshold is then too high and the row is done again).
+    if (nvec > SAMPLE_VECS) {
+        // A row much longer than the sample: every thread takes the largest of its 32 sampled
+        // logits, and the r-th largest of these 256 maxima stands in for the r-th largest of the
+        // sample.  It is never above it (the maxima are r different sampled logits), so the
+        // threshold only gets safer, and a little lower when two of the sample's best share a
+        // thread; one key per thread makes the passes cheap.
+        float mx = L::vmax(sv[0]);
+#pragma unroll
+        for (int i = 1; i < SEL_SAMPLE; ++i) mx = fmaxf(mx, L::vmax(sv[i]));
+        const uint32_t key = order_key(mx);
+        if (tid == 0) ctl.remaining = min(r, unsigned(TOPM_THREADS));
 #pragma unroll 1
-    for (int shift = 24; shift >= (DT == DISC_BF16 ? 16 : 0); shift -= 8) {
-        rs.hist[tid] = 0u;
-        __syncthreads();
-        const uint32_t prefix = ctl.prefix;
+        for (int shift = 24; shift >= (DT == DISC_BF16 ? 16 : 0); shift -= 8) {
+            rs.hist[tid] = 0u;
+            __syncthreads();
+            const uint32_t prefix = ctl.prefix;
+            if (shift == 24 || (key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&rs.hist[(key >> shift) & 255u], 1u);
+            __syncthreads();
+            pick_bin256(rs.hist, prefix, shift, rs.wsum, &ctl.prefix, &ctl.remaining, &ctl.ties);
+        }
+    } else {
+        // The r-th largest key of the sample, eight bits at a time.  The -inf that stands for "past the
+        // end of the row" has the lowest key of all numbers and r counts real logits only, so the
+        // fill never matters.  bf16: the two 16-bit keys of a word are formed together, and a NaN
+        // counts as a large value here (the threshold is then too high and the row is done again).
+#pragma unroll 1
+        for (int shift = 24; shift >= (DT == DISC_BF16 ? 16 : 0); shift -= 8) {
+            rs.hist[tid] = 0u;
+            __syncthreads();
+            const uint32_t prefix = ctl.prefix;
 #pragma unroll
-        for (int i = 0; i < SEL_SAMPLE; ++i) {
-            if (DT == DISC_BF16) {
-                const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
+            for (int i = 0; i < SEL_SAMPLE; ++i) {
+                if (DT == DISC_BF16) {
+                    const uint32_t w[4] = {sv[i].x, sv[i].y, sv[i].z, sv[i].w};
 #pragma unroll
-                for (int j = 0; j < 4; ++j) {
-                    const uint32_t neg = (w[j] & 0x80008000u) >> 15;             // 1 in the halves that are negative
-                    const uint32_t k2 = w[j] ^ ((neg * 0xFFFFu) | 0x80008000u);  // ~h there, h ^ 0x8000 elsewhere
-                    const uint32_t ka = k2 & 0xFFFFu, kb = k2 >> 16;
-                    if (shift == 24) {
-                        atomicAdd(&rs.hist[ka >> 8], 1u);
-                        atomicAdd(&rs.hist[kb >> 8], 1u);
-                    } else {
-                        if ((ka >> 8) == (prefix >> 24)) atomicAdd(&rs.hist[ka & 255u], 1u);
-                        if ((kb >> 8) == (prefix >> 24)) atomicAdd(&rs.hist[kb & 255u], 1u);
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t neg = (w[j] & 0x80008000u) >> 15;             // 1 in the halves that are negative
+                        const uint32_t k2 = w[j] ^ ((neg * 0xFFFFu) | 0x80008000u);  // ~h there, h ^ 0x8000 elsewhere
+                        const uint32_t ka = k2 & 0xFFFFu, kb = k2 >> 16;
+                        if (shift == 24) {
+                            atomicAdd(&rs.hist[ka >> 8], 1u);
+                            atomicAdd(&rs.hist[kb >> 8], 1u);
+                        } else {
+                            if ((ka >> 8) == (prefix >> 24)) atomicAdd(&rs.hist[ka & 255u], 1u);
+                            if ((kb >> 8) == (prefix >> 24)) atomicAdd(&rs.hist[kb & 255u], 1u);
+                        }
+                    }
+                } else {
+                    float x[EPV];
+                    L::unpack(sv[i], x);
+#pragma unroll
+                    for (int j = 0; j < EPV; ++j) {
+                        const uint32_t key = order_key(x[j]);
+                        if (shift == 24 || (key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&rs.hist[(key >> shift) & 255u], 1u);
                     }
                 }
-            } else {
-                float x[EPV];
-                L::unpack(sv[i], x);
-#pragma unroll
-                for (int j = 0; j < EPV; ++j) {
-                    const uint32_t key = order_key(x[j]);
-                    if (shift == 24 || (key >> (shift + 8)) == (prefix >> (shift + 8))) atomicAdd(&rs.hist[(key >> shift) & 255u], 1u);
-                }
             }
+            __syncthreads();
+            pick_bin256(rs.hist, prefix, shift, rs.wsum, &ctl.prefix, &ctl.remaining, &ctl.ties);
         }
-        __syncthreads();
-        pick_bin256(rs.hist, prefix, shift, rs.wsum, &ctl.prefix, &ctl.remaining, &ctl.ties);
     }
     // a logit is a candidate if it is at least this (a NaN key: no threshold, every logit is one)
     float thr = -CUDART_INF_F;
