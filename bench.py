@@ -500,11 +500,13 @@ def fused_projection(disc, G, lm, ctx, w, dev, L, seed, reps=3):
     logits = torch.empty((R, w.V), dtype=torch.bfloat16, device=dev)
     seq = torch.empty((R, G.l_max), dtype=torch.int32, device=dev)
     out = disc.StepOutputs.empty(R, dev)
-    peak_tf = None
+    peak_tf = peak_sus = None
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(path):
         with open(path) as f:
-            peak_tf = float(json.load(f).get("bf16_tflops", 0)) or None
+            peaks = json.load(f)
+            peak_tf = float(peaks.get("bf16_tflops", 0)) or None
+            peak_sus = float(peaks.get("bf16_tflops_sustained", 0)) or None
 
     def decode(fused_path):
         ms = np.zeros(L)
@@ -545,6 +547,9 @@ def fused_projection(disc, G, lm, ctx, w, dev, L, seed, reps=3):
     res["roofline"] = {"bound": "tensor", "kernel": "disc_project_pair_kernel (+ tile flags + step)", "achieved": round(tf, 1),
                        "peak": peak_tf, "unit": "TFLOP/s", "frac": None if not peak_tf else round(tf / peak_tf, 4),
                        "peak_kind": "of measured (cuBLAS bf16 burst)" if peak_tf else "unavailable",
+                       # the positions are timed one after the other inside decodes that keep the GPU at its
+                       # power cap, which is what the sustained figure of the same library GEMM describes
+                       "peak_sustained": peak_sus, "frac_of_sustained": None if not peak_sus else round(tf / peak_sus, 4),
                        "traffic": None}
     # end to end through the fused call: every position's hidden vectors start in pinned host memory
     # (R x d bf16 instead of R x V logits), the chosen sequences are read back at the end
