@@ -446,6 +446,15 @@ def run_ours(args):
                                "dead_end_rows": int((outp.status == 1).sum().item())})
         mask_stress["verify_top_m"] = verify
 
+    # ---- a whole decode in the paper's top-M mode next to the exact-mask decode (secondary figure)
+    topm_decode = None
+    if rank == 0 and w.name == "large" and not args.no_fused:
+        try:
+            topm_decode = top_m_decode(disc, G, lm, ctx, w, dev, L, seed)
+        except Exception as e:                     # a secondary figure never fails the line
+            topm_decode = {"error": repr(e)[:200]}
+        torch.cuda.empty_cache()
+
     # ---- the projection fused with the step (secondary figure): a free-running decode per variant,
     # an event pair around every position; the unfused variant is torch's matmul + disc_step
     fused = None
@@ -480,7 +489,7 @@ def run_ours(args):
                                   "(source of the roofline's per-launch times)", "clocks": clocks},
                 "deterministic_replay": same_tokens,
                 "lm_projection_ms_per_position": round(lm_ms, 3), "mask_stress": mask_stress,
-                "fused_projection": fused,
+                "fused_projection": fused, "top_m_decode": topm_decode,
                 "set": {"members": G.N, "entries": G.E, "index_nodes": G.n_nodes,
                         "device_mb": round(G.device_bytes / 1e6, 1), "build_s": round(G.build_seconds, 3)},
                 "setup_s": round(time.time() - t_setup, 1)}
@@ -488,6 +497,59 @@ def run_ours(args):
     G.close()
     if use_dist:
         dist.destroy_process_group()
+
+
+def top_m_decode(disc, G, lm, ctx, w, dev, L, seed, M=50, bonus=8.0, reps=5):
+    """Secondary figure: a whole decode in the paper's top-M mode (DiscDecoder(top_m=M)), next to the
+    exact-mask decode of the same logits.  The stand-in model knows nothing of the set, so its top-M
+    tokens are almost never valid after the first position; a model trained for the task puts its
+    mass on valid tokens.  The logits used here stand in for such a model: the stand-in's logits with
+    `bonus` added to every valid next token (the valid sets come from disc_mask, outside the timed
+    region).  Both decodes replay the same recorded logits as one CUDA graph each."""
+    import torch
+    R = w.R
+    rec = disc.DiscDecoder(G, w.B, w.K, dev, top_m=M)
+    rec.reset()
+    prev = ctx.to(dev, torch.int64).repeat_interleave(w.K)
+    shifts = torch.arange(32, device=dev, dtype=torch.int32)
+    steps = []
+    for t in range(L):
+        z = lm.logits(prev)
+        m = disc.disc_mask(G, rec.seq, rec.state.depth)["mask"]
+        for r0 in range(0, R, 512):                               # in slices: the unpacked bits are 32 x the mask
+            bits = ((m[r0:r0 + 512].unsqueeze(-1) >> shifts) & 1).reshape(min(512, R - r0), -1)[:, :w.V]
+            z[r0:r0 + 512] += (bits * bonus).to(z.dtype)
+        steps.append(z)
+        o = rec.step(z, t, seed=seed)
+        prev = torch.where(o.token >= 0, o.token.to(torch.int64), prev)
+    rec.finish(seed=seed)
+    torch.cuda.synchronize()
+    tokens_topm = int((rec.seq >= 0).sum().item())
+    dead = int(torch.isinf(rec.state.logw).sum().item())
+
+    def timed(decoder):
+        graph = decoder.capture(steps, seed=seed)
+        for _ in range(2):
+            graph.replay()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            graph.replay()
+        b.record()
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
+
+    ms_topm = timed(rec)
+    exact = disc.DiscDecoder(G, w.B, w.K, dev)
+    ms_exact = timed(exact)
+    tokens_exact = int((exact.seq >= 0).sum().item())
+    return {"M": M, "bonus_on_valid_tokens": bonus,
+            "top_m": {"ms_per_decode": round(ms_topm, 4), "tokens_per_decode": tokens_topm,
+                      "tokens_per_s": round(tokens_topm / (ms_topm * 1e-3), 1), "dead_end_rows": dead},
+            "exact_mask": {"ms_per_decode": round(ms_exact, 4), "tokens_per_decode": tokens_exact,
+                           "tokens_per_s": round(tokens_exact / (ms_exact * 1e-3), 1)},
+            "note": "same logits for both decodes (stand-in logits + bonus on the valid next tokens of the top-M "
+                    "decode's own prefixes); each decode replayed as one CUDA graph"}
 
 
 def fused_projection(disc, G, lm, ctx, w, dev, L, seed, reps=3):
