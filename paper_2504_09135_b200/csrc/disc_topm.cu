@@ -326,6 +326,14 @@ struct Lane<DISC_BF16> {
         const uint32_t w = *reinterpret_cast<const uint32_t*>(&c);
         return fmaxf(__uint_as_float(w << 16), __uint_as_float(w & 0xffff0000u));
     }
+    // does any element reach thr (a value of the row's own type)?  Packed: three maxima and one
+    // comparison of both halves; a vector of NaNs counts as reaching it, which costs a look at it
+    // later and nothing else.
+    __device__ static __forceinline__ bool reaches(const uint4& v, float thr) {
+        const __nv_bfloat162 a = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.x), *reinterpret_cast<const __nv_bfloat162*>(&v.y));
+        const __nv_bfloat162 b = __hmax2(*reinterpret_cast<const __nv_bfloat162*>(&v.z), *reinterpret_cast<const __nv_bfloat162*>(&v.w));
+        return !__hblt2(__hmax2(a, b), __float2bfloat162_rn(thr));
+    }
     // elements id0 .. id0+7 read one by one; -inf where the row has ended
     __device__ static __forceinline__ uint4 gather(const void* rowp, int id0, int V) {
         uint32_t w[4];
@@ -348,6 +356,7 @@ struct Lane<DISC_F32> {
     __device__ static __forceinline__ float vmax(const uint4& v) {
         return fmaxf(fmaxf(__uint_as_float(v.x), __uint_as_float(v.y)), fmaxf(__uint_as_float(v.z), __uint_as_float(v.w)));
     }
+    __device__ static __forceinline__ bool reaches(const uint4& v, float thr) { return vmax(v) >= thr; }
     __device__ static __forceinline__ uint4 gather(const void* rowp, int id0, int V) {
         uint32_t w[4];
         const uint32_t* r = static_cast<const uint32_t*>(rowp);
@@ -639,7 +648,7 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
             acc1 = __fadd2_rn(acc1, make_float2(ex2_approx(y1.x), ex2_approx(y1.y)));
         }
         }
-        if (L::vmax(raw) >= thr) {
+        if (L::reaches(raw, thr)) {
             const unsigned int pos = atomicAdd(&ctl.count, 1u);
             if (pos < unsigned(SEL_HITS)) hits[pos] = vi;
         }
