@@ -459,13 +459,17 @@ __device__ __noinline__ void select_best(uint32_t* keys, int32_t* ids, unsigned 
     // passed, nobody reads the histogram any more), then moved to the front
     uint32_t* tk = hist;
     int32_t* ti = reinterpret_cast<int32_t*>(hist + SEL_KEEP);
-    for (unsigned int i = tid; i < cnt; i += TOPM_THREADS) {
-        const uint32_t k = keys[i], km = k & key_mask;
-        const int32_t id = ids[i];
-        if (km > thr_key || (km == thr_key && id <= id_thr)) {
-            const unsigned int pos = atomicAdd(&c.kept, 1u);
-            if (pos < unsigned(SEL_KEEP)) { tk[pos] = k; ti[pos] = id; }
-        }
+    for (unsigned int i0 = 0; i0 < cnt; i0 += TOPM_THREADS) {             // the lanes of a warp stay together
+        const unsigned int i = i0 + tid;
+        const uint32_t k = i < cnt ? keys[i] : 0u, km = k & key_mask;
+        const int32_t id = i < cnt ? ids[i] : 0;
+        const bool keep = i < cnt && (km > thr_key || (km == thr_key && id <= id_thr));
+        const uint32_t ballot = __ballot_sync(FULL, keep);                // one reservation per warp
+        const int lane = tid & 31;
+        unsigned int base = 0u;
+        if (lane == 0 && ballot) base = atomicAdd(&c.kept, unsigned(__popc(ballot)));
+        const unsigned int pos = __shfl_sync(FULL, base, 0) + unsigned(__popc(ballot & ((1u << lane) - 1u)));
+        if (keep && pos < unsigned(SEL_KEEP)) { tk[pos] = k; ti[pos] = id; }
     }
     __syncthreads();
     const unsigned int n_kept = min(c.kept, unsigned(SEL_KEEP));      // = want
@@ -626,9 +630,11 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
 
     // ---- B. one pass over the row: the sum for the log-sum-exp, and the vectors that hold a candidate
     // (a vector is tested as a whole; what it holds is looked at in C).  No barriers: thread t
-    // takes the vectors t, t+256, ... with SEL_U loads in flight.
-    auto consume = [&](const uint4& raw, int vi) {
-        if (attempt == 0) {
+    // takes the vectors t, t+256, ... with SEL_U loads in flight.  Which of its vectors reach the
+    // threshold a thread keeps as bits in a register and writes to the list every 64 vectors: inside
+    // the loop a hit then costs a predicated OR, not a branch that most warps would take at large M.
+    auto add_to_sum = [&](const uint4& raw) {
+        if (attempt != 0) return;
         float x[EPV];
         L::unpack(raw, x);
         if (!touched) {
@@ -647,22 +653,58 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
             acc0 = __fadd2_rn(acc0, make_float2(ex2_approx(y0.x), ex2_approx(y0.y)));
             acc1 = __fadd2_rn(acc1, make_float2(ex2_approx(y1.x), ex2_approx(y1.y)));
         }
-        }
-        if (L::reaches(raw, thr)) {
-            const unsigned int pos = atomicAdd(&ctl.count, 1u);
-            if (pos < unsigned(SEL_HITS)) hits[pos] = vi;
-        }
+    };
+    auto note = [&](int vi) {
+        const unsigned int pos = atomicAdd(&ctl.count, 1u);
+        if (pos < unsigned(SEL_HITS)) hits[pos] = vi;
     };
     {
-        int vi = tid;
-        for (; vi + (SEL_U - 1) * TOPM_THREADS < nvec; vi += SEL_U * TOPM_THREADS) {
-            uint4 raw[SEL_U];
+        static_assert(64 % SEL_U == 0, "whole batches per 64-bit word");
+        constexpr int BATCHES = 64 / SEL_U;          // batches of SEL_U vectors per word of hit bits
+        // whole batches (the same number for every thread of the block), then the few vectors left
+        const int n_batches = nvec / (SEL_U * TOPM_THREADS);
+        for (int b0 = 0; b0 < n_batches; b0 += BATCHES) {
+            const int vi0 = tid + b0 * SEL_U * TOPM_THREADS;
+            const int nb = min(BATCHES, n_batches - b0);
+            unsigned long long bits = 0ull;
+#pragma unroll 1
+            for (int it = 0; it < nb; ++it) {
+                const int vi = vi0 + it * SEL_U * TOPM_THREADS;
+                uint4 raw[SEL_U];
 #pragma unroll
-            for (int u = 0; u < SEL_U; ++u) raw[u] = load_vec(vi + u * TOPM_THREADS);
+                for (int u = 0; u < SEL_U; ++u) raw[u] = load_vec(vi + u * TOPM_THREADS);
+                unsigned int m = 0u;
 #pragma unroll
-            for (int u = 0; u < SEL_U; ++u) consume(raw[u], vi + u * TOPM_THREADS);
+                for (int u = 0; u < SEL_U; ++u) {
+                    add_to_sum(raw[u]);
+                    m |= L::reaches(raw[u], thr) ? (1u << u) : 0u;
+                }
+                bits |= static_cast<unsigned long long>(m) << (it * SEL_U);
+            }
+            // the warp's hits go to the list with one reservation (the lanes are together here: the
+            // loop above runs the same number of times in every thread)
+            const unsigned int mine = unsigned(__popcll(bits));
+            unsigned int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int v = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += v;
+            }
+            unsigned int base = 0u;
+            if (lane == 31 && incl) base = atomicAdd(&ctl.count, incl);
+            unsigned int pos = __shfl_sync(FULL, base, 31) + incl - mine;
+            while (bits) {                            // bit it*SEL_U + u: vector vi0 + (it*SEL_U + u) * 256
+                const int bpos = __ffsll(static_cast<long long>(bits)) - 1;
+                bits &= bits - 1ull;
+                if (pos < unsigned(SEL_HITS)) hits[pos] = vi0 + bpos * TOPM_THREADS;
+                ++pos;
+            }
         }
-        for (; vi < nvec; vi += TOPM_THREADS) consume(load_vec(vi), vi);
+        for (int vi = tid + n_batches * SEL_U * TOPM_THREADS; vi < nvec; vi += TOPM_THREADS) {
+            const uint4 raw = load_vec(vi);
+            add_to_sum(raw);
+            if (L::reaches(raw, thr)) note(vi);
+        }
     }
 
     // ---- the row's sum over the whole vocabulary
@@ -735,15 +777,30 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
     __syncthreads();
     bool redo = n_hits > unsigned(SEL_HITS), too_few = false;
     if (!redo) {
-        for (unsigned int h = tid; h < n_hits; h += TOPM_THREADS) {
-            const int vi = hits[h];
+        for (unsigned int h0 = 0; h0 < n_hits; h0 += TOPM_THREADS) {      // the lanes of a warp stay together
+            const unsigned int h = h0 + tid;
+            const int vi = h < n_hits ? hits[h] : 0;
             float x[EPV];
             L::unpack(load_vec(vi), x);
+            unsigned int take = 0u;                       // which of the vector's logits are candidates
+#pragma unroll
+            for (int j = 0; j < EPV; ++j) take |= (h < n_hits && vi * EPV + j < V && x[j] >= thr) ? (1u << j) : 0u;
+            // one reservation per warp
+            const unsigned int mine = unsigned(__popc(take));
+            unsigned int incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned int v = __shfl_up_sync(FULL, incl, o);
+                if (lane >= o) incl += v;
+            }
+            unsigned int base = 0u;
+            if (lane == 31 && incl) base = atomicAdd(&ctl.count, incl);
+            unsigned int pos = __shfl_sync(FULL, base, 31) + incl - mine;
 #pragma unroll
             for (int j = 0; j < EPV; ++j) {
-                if (vi * EPV + j < V && x[j] >= thr) {
-                    const unsigned int pos = atomicAdd(&ctl.count, 1u);
+                if ((take >> j) & 1u) {
                     if (pos < unsigned(SEL_CAP)) { keys[pos] = order_key(x[j]); ids[pos] = vi * EPV + j; }
+                    ++pos;
                 }
             }
         }
@@ -758,35 +815,61 @@ __global__ void __launch_bounds__(TOPM_THREADS, DISC_TOPM_BLOCKS) disc_topm_stre
                 n = ctl.count;
             }
             // the ids in ascending order: few - every thread counts the ids below its own; many - a
-            // bitonic network over the next power of two
+            // counting sort over the ids' upper eleven bits, then order inside the (tiny) buckets
             __syncthreads();
-            int32_t* tids = reinterpret_cast<int32_t*>(rs.hist);
+            const int32_t* tids;
             if (n <= unsigned(TOPM_THREADS)) {
+                int32_t* dst = reinterpret_cast<int32_t*>(rs.hist);
                 if (unsigned(tid) < n) {
                     const int32_t mine = ids[tid];
                     unsigned int below = 0u;
                     for (unsigned int j = 0; j < n; ++j) below += ids[j] < mine ? 1u : 0u;
-                    tids[below] = mine;
+                    dst[below] = mine;
                 }
+                tids = dst;
                 __syncthreads();
             } else {
-                unsigned int P = 1u;
-                while (P < n) P <<= 1;
-                for (unsigned int i = tid; i < P; i += TOPM_THREADS) tids[i] = i < n ? ids[i] : 0x7fffffff;
+                const int shift = max(32 - __clz(V - 1) - RADIX_BITS, 0);      // id >> shift < BINS
+                unsigned int* cnt = rs.hist;
+                int32_t* dst = reinterpret_cast<int32_t*>(keys);               // the keys have done their work
+                for (int i = tid; i < BINS; i += TOPM_THREADS) cnt[i] = 0u;
                 __syncthreads();
-                for (unsigned int k = 2u; k <= P; k <<= 1) {
-                    for (unsigned int j = k >> 1; j > 0u; j >>= 1) {
-                        for (unsigned int i = tid; i < P; i += TOPM_THREADS) {
-                            const unsigned int l = i ^ j;
-                            if (l > i) {
-                                const int32_t a = tids[i], c = tids[l];
-                                const bool up = (i & k) == 0u;
-                                if ((a > c) == up) { tids[i] = c; tids[l] = a; }
-                            }
-                        }
-                        __syncthreads();
+                for (unsigned int i = tid; i < n; i += TOPM_THREADS) atomicAdd(&cnt[ids[i] >> shift], 1u);
+                __syncthreads();
+                // exclusive prefix sums over the buckets: thread t owns the buckets [8t, 8t+8)
+                unsigned int len[BINS_PER_THREAD], mine = 0u;
+#pragma unroll
+                for (int k = 0; k < BINS_PER_THREAD; ++k) { len[k] = cnt[tid * BINS_PER_THREAD + k]; mine += len[k]; }
+                unsigned int incl = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const unsigned int v = __shfl_up_sync(FULL, incl, o);
+                    if (lane >= o) incl += v;
+                }
+                if (lane == 31) rs.wsum[warp] = incl;
+                __syncthreads();
+                unsigned int start = incl - mine;
+                for (int w2 = 0; w2 < warp; ++w2) start += rs.wsum[w2];
+                unsigned int first[BINS_PER_THREAD];
+#pragma unroll
+                for (int k = 0; k < BINS_PER_THREAD; ++k) { first[k] = start; cnt[tid * BINS_PER_THREAD + k] = start; start += len[k]; }
+                __syncthreads();
+                for (unsigned int i = tid; i < n; i += TOPM_THREADS) {
+                    const int32_t id = ids[i];
+                    dst[atomicAdd(&cnt[id >> shift], 1u)] = id;
+                }
+                __syncthreads();
+#pragma unroll
+                for (int k = 0; k < BINS_PER_THREAD; ++k) {
+                    for (unsigned int i = first[k] + 1u; i < first[k] + len[k]; ++i) {      // insertion sort of a bucket
+                        const int32_t v = dst[i];
+                        unsigned int j = i;
+                        for (; j > first[k] && dst[j - 1] > v; --j) dst[j] = dst[j - 1];
+                        dst[j] = v;
                     }
                 }
+                tids = dst;
+                __syncthreads();
             }
             for (int m = tid; m < p.M; m += TOPM_THREADS) out[m] = unsigned(m) < n ? tids[m] : -1;
         }
