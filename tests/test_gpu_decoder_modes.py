@@ -89,3 +89,21 @@ def test_decode_from_hidden_vectors_ends_every_row_in_a_member():
                                                                    lm.projection_rows(), 0)
     finally:
         G.close()
+
+
+def test_top_m_decode_replayed_as_a_graph_gives_the_same_result():
+    w, G, lm, ctx, _ = _setup("genret", B=16, K=8)
+    try:
+        dec = disc.DiscDecoder(G, w.B, w.K, DEV, top_m=128)
+        keep = []
+        dec.decode(lm, ctx, seed=9, keep_logits=keep)
+        torch.cuda.synchronize()
+        seq, logw, idx = dec.seq.clone(), dec.state.logw.clone(), dec.res["idx"].clone()
+        graph = dec.capture(keep, seed=9)
+        dec.seq.fill_(-7)
+        graph.replay()
+        torch.cuda.synchronize()
+        assert torch.equal(dec.seq, seq) and torch.equal(dec.res["idx"], idx)
+        assert torch.equal(dec.state.logw, logw)
+    finally:
+        G.close()
