@@ -110,7 +110,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, volati
     *abort = 1;
     return false;
 }
-// the same for a whole warp that must stay converged: lane 0 waits, the others follow its verdict
+// the same for a whole warp that must stay converged: lane 0 waits, the others take over its result
 // and then observe the completed phase themselves
 __device__ __forceinline__ bool mbar_wait_warp(uint64_t* bar, uint32_t parity, volatile int* abort, int lane) {
     int ok = 1;

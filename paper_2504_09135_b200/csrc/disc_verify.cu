@@ -107,7 +107,7 @@ __device__ __forceinline__ RowRange row_range(const VerifyParams& p, int64_t i) 
 __device__ __forceinline__ int32_t key_at(const VerifyParams& p, int32_t j, int32_t d) {
     return __ldg(p.tok + __ldg(p.row_off + j) + d);
 }
-// the first row of [x, y) whose key is not below t (y if there is none), then the verdict
+// the first row of [x, y) whose key is not below t (y if there is none), then what the search says
 __device__ __forceinline__ void finish_candidate(const VerifyParams& p, const RowRange& r, int64_t i, int64_t g, int32_t t,
                                                  int32_t x, int32_t y) {
     while (x < y) {
