@@ -8,10 +8,15 @@
 // writes, however they were overlapped).  Writing the packed mask row (Section 2.1's valid set of
 // the node reached: a copy of a prebuilt row for the empty prefix and for nodes with many
 // children, otherwise zeros with the children's bits merged in) is 16 KB of stores that need no
-// answer, and HBM takes them fastest from few warps that each stream a whole row (on B200, rows of
-// zeros: eight writing warps per SM reach 6.7 TB/s, forty reach 5.7).
+// answer, and HBM takes them fastest when the rows in flight are few and neighbours (see the
+// second half of this file).
 //
-// One kernel does both, one block per SM, in rounds of two phases:
+// Rows of at least 128 bytes that are 16-byte aligned and a multiple of 16 bytes long (the large
+// vocabularies): two kernels, disc_mask_walk_kernel (every walk, one thread per prefix) and disc_mask_team_kernel
+// (the rows, by teams of warps that draw row indices from one counter); they are described where
+// they stand.
+//
+// Other rows: one kernel, one block per SM, in rounds of two phases:
 //   1. every warp draws up to 32 rows from a global counter and walks their prefixes, one THREAD
 //      per prefix, all walks of the GPU in flight at once.  Range, cursor and status go out; a
 //      128-byte descriptor (row, node, child range, which prebuilt row to copy, the first
@@ -22,8 +27,7 @@
 //      list too long for the descriptor is staged there by asynchronous copies while the previous
 //      row is written; a heavy node's prebuilt row is copied from L2 (or staged likewise when the
 //      staging buffer is built large enough to hold a row).
-// All blocks start together, so the phases line up across the GPU: a burst of reads, then a pure
-// write stream.  There are no waits other than block barriers.
+// There are no waits other than block barriers.
 //
 // Calls that ask for no mask (ranges, cursor and status only) run the walks alone.
 //
@@ -506,6 +510,334 @@ __global__ void __launch_bounds__(FUSED_THREADS, 1) disc_mask_kernel(const MaskP
     }
 }
 
+
+// ---- two kernels: every walk first, then the rows in the order of their indices ------------------------
+// HBM takes a stream of 16 KB rows fastest when the rows being written at any moment are neighbours
+// and few: on B200, rows of zeros drawn one by one from a global counter reach 7.2-7.3 TB/s with four
+// to six rows in flight per SM (600-900 on the GPU), 4.5 TB/s with eight or more, and 6.1 TB/s when
+// every SM works through a share of its own, whatever the order inside it.  So the rows are written
+// by TEAMS of warps (a row's 512-byte spans dealt out among the team's warps: enough warps to
+// generate the rows, few rows in flight), every team drawing the next row index from one counter.
+// That needs every prefix's walk done before the first row is written, so the walks are a kernel
+// of their own (one thread per prefix, all of them in flight at once while DRAM has nothing else to
+// do), which parks what the writer needs - node, child range, which prebuilt row to copy, the
+// first 27 children - in the first 128 bytes of the prefix's own mask row, to be read back by the
+// team (from L2) before it overwrites them.  Rows shorter than that, and rows that are not 16-byte
+// aligned, take the one-kernel path above.
+#ifndef DISC_MASK_TEAM
+#define DISC_MASK_TEAM 4
+#endif
+#ifndef DISC_MASK_TEAMS
+#define DISC_MASK_TEAMS 6
+#endif
+constexpr int TEAM = DISC_MASK_TEAM;             // warps that write one row together
+constexpr int TEAMS = DISC_MASK_TEAMS;           // rows in flight per SM
+constexpr int TEAM_THREADS = 32 * TEAM * TEAMS;
+static_assert(TEAMS <= 15, "one named barrier per team");
+constexpr int WALK_THREADS = 256;
+
+__global__ void __launch_bounds__(WALK_THREADS) disc_mask_walk_kernel(const MaskParams p) {
+    const int64_t i = int64_t(blockIdx.x) * WALK_THREADS + threadIdx.x;
+    if (i >= p.n) return;
+    const int32_t len = __ldg(p.prefix_len + i);
+    const int32_t* pre = p.prefix + i * p.prefix_ld;
+    bool ok = (len >= 0 && len <= p.prefix_ld && len <= p.l_max);     // no member is longer than l_max
+    int32_t node = 0, lo = 0, hi = p.N, cb = 0, ce = 0;
+    if (ok) { cb = __ldg(p.child_begin); ce = __ldg(p.child_begin + 1); }
+    int32_t t_next = (ok && len > 0) ? __ldg(pre) : 0;
+    for (int32_t d = 0; ok && d < len; ++d) {
+        const int32_t t = t_next;
+        if (d + 1 < len) t_next = __ldg(pre + d + 1);        // fetched while this level is searched
+        if (t < 0 || t >= p.V) { ok = false; break; }
+        if (node == 0) {
+            const int32_t k = __ldg(p.root_child + t);
+            if (k < 0) { ok = false; break; }
+            lo = __ldg(p.node_lo + k);
+            if (k + 1 < ce) hi = __ldg(p.node_lo + k + 1);
+            node = k;
+            cb = __ldg(p.child_begin + k);
+            ce = __ldg(p.child_begin + k + 1);
+        } else {
+            const ChildInfo c = find_child_info(p.node_tok, p.node_lo, p.child_begin, cb, ce, t);
+            if (c.k < 0) { ok = false; break; }
+            lo = c.lo;
+            if (c.k + 1 < ce) hi = c.lo_next;
+            node = c.k;
+            cb = c.cb;
+            ce = c.ce;
+        }
+    }
+    if (p.lo_out) p.lo_out[i] = ok ? lo : -1;
+    if (p.hi_out) p.hi_out[i] = ok ? hi : -1;
+    if (p.node_out) p.node_out[i] = ok ? node : -1;
+    p.status_out[i] = ok ? 0 : DISC_ROW_DEAD;
+    // the descriptor: node (-1: dead), child range, prebuilt row (-2 none, -1 the root's, -3 a heavy
+    // node's: the writer looks up which), a spare word, the first DESC_TOKENS children
+    uint32_t dsc[DESC_WORDS];
+    int32_t sel = -2;
+    if (!ok) { cb = 0; ce = 0; }
+    else if (node == 0) sel = -1;
+    else if (ce - cb > DISC_HEAVY_MIN) sel = -3;
+    dsc[0] = uint32_t(ok ? node : -1); dsc[1] = uint32_t(cb); dsc[2] = uint32_t(ce); dsc[3] = uint32_t(sel); dsc[4] = 0u;
+    const int32_t m = sel == -2 ? min(ce - cb, DESC_TOKENS) : 0;
+#pragma unroll
+    for (int j0 = 0; j0 < DESC_TOKENS; j0 += 9) {
+#pragma unroll
+        for (int u = 0; u < 9; ++u) dsc[5 + j0 + u] = (j0 + u < m) ? uint32_t(__ldg(p.node_tok + cb + j0 + u)) : 0u;
+    }
+    // parked with the request that L2 keep the lines: they are read back while a gigabyte of mask
+    // rows streams through L2 (stored "evict first"), and a descriptor that had to come back from
+    // DRAM would be a read in the middle of the write stream
+    uint4* head = reinterpret_cast<uint4*>(p.mask_out + size_t(i) * p.W);
+    const uint64_t keep = l2_policy_evict_last();
+#pragma unroll
+    for (int q = 0; q < DESC_WORDS / 4; ++q) {
+        asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(head + q), "r"(dsc[4 * q]), "r"(dsc[4 * q + 1]),
+                     "r"(dsc[4 * q + 2]), "r"(dsc[4 * q + 3]), "l"(keep)
+                     : "memory");
+    }
+}
+
+__device__ __forceinline__ void team_barrier(int team) {
+    asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(TEAM * 32) : "memory");
+}
+
+// What a team knows of a row from its parked descriptor (the same in every lane of every warp).
+struct TeamRow {
+    int32_t node, cb, ce, sel;     // sel: -2 no prebuilt row, -1 the root's, -3 a heavy node's
+    int32_t tk;                    // lane l: child l of the row (l < DESC_TOKENS)
+    int kind;                      // 0: written straight from the descriptor (or the root's row), 1: a heavy
+                                   // node's prebuilt row, 2: more children than the descriptor holds
+};
+__device__ __forceinline__ TeamRow team_row(uint32_t word, int lane) {
+    TeamRow r;
+    r.node = int32_t(__shfl_sync(FULL, word, 0));
+    r.cb = int32_t(__shfl_sync(FULL, word, 1));
+    r.ce = int32_t(__shfl_sync(FULL, word, 2));
+    r.sel = int32_t(__shfl_sync(FULL, word, 3));
+    r.tk = int32_t(__shfl_sync(FULL, word, (lane + 5) & 31));
+    r.kind = r.sel == -3 ? 1 : ((r.sel == -2 && r.node >= 0 && r.ce - r.cb > DESC_TOKENS) ? 2 : 0);
+    return r;
+}
+
+// Rows of kind 1 and 2 are put together in the team's buffer in shared memory (bm: a whole mask
+// row; ts: up to DISC_HEAVY_MIN child tokens) and streamed out from there.  prepare_row starts that
+// a row ahead: asynchronous copies of the prebuilt row, or of the child list (and the buffer is
+// zeroed for the bits to come).  Warp h of the team, thread tt of its TEAM*32.
+__device__ __forceinline__ void prepare_row(const MaskParams& p, const TeamRow& r, uint32_t* bm, uint32_t* ts, int h, int lane) {
+    const int n4 = p.W >> 2;
+    const int tt = h * 32 + lane;
+    if (r.kind == 1) {
+        const int32_t hv = warp_heavy_index(p.heavy_nodes, p.n_heavy, r.node, lane);
+        if (hv >= 0) {
+            const uint4* src4 = reinterpret_cast<const uint4*>(p.heavy_masks + size_t(hv) * p.Wp);
+            for (int w = tt; w < n4; w += TEAM * 32) cp_async16(reinterpret_cast<uint4*>(bm) + w, src4 + w);
+        } else {                         // cannot happen for a consistent set: an empty row
+            for (int w = tt; w < n4; w += TEAM * 32) reinterpret_cast<uint4*>(bm)[w] = make_uint4(0u, 0u, 0u, 0u);
+        }
+    } else {
+        const int nc = r.ce - r.cb;
+        for (int j = tt; j < nc; j += TEAM * 32) cp_async4(ts + j, p.node_tok + r.cb + j);
+        for (int w = tt; w < n4; w += TEAM * 32) reinterpret_cast<uint4*>(bm)[w] = make_uint4(0u, 0u, 0u, 0u);
+    }
+}
+
+// The share of warp h of a team in one mask row: the spans it with it % TEAM == h (a span = 32
+// 16-byte vectors = 4,096 tokens).  bm/ts: the team's buffers (null when a row does not fit them:
+// rows of kind 1 and 2 are then generated span by span from global memory); prepared: prepare_row
+// has run for this row.  Every warp of the team takes the same path (it contains team barriers).
+__device__ __forceinline__ void write_row_team(const MaskParams& p, int64_t i, const TeamRow& r, int team, int h,
+                                               const uint32_t* s_root, uint32_t* bm, uint32_t* ts, bool prepared,
+                                               uint32_t* patch, uint64_t keep, int lane) {
+    const uint4 z = make_uint4(0u, 0u, 0u, 0u);
+    const int nc = r.ce - r.cb;
+    uint4* row4 = reinterpret_cast<uint4*>(p.mask_out + size_t(i) * p.W);
+    const int n4 = p.W >> 2;
+    const int n_it = (n4 + 31) >> 5;
+    if (r.kind != 0 && bm) {
+        if (!prepared) prepare_row(p, r, bm, ts, h, lane);
+        cp_async_wait_all();
+        team_barrier(team);                          // the copies and the zeros of all four warps are in place
+        if (r.kind == 2) {
+            for (int j = h * 32 + lane; j < nc; j += TEAM * 32) {
+                const uint32_t t = ts[j];
+                atomicOr(&bm[t >> 5], 1u << (t & 31));
+            }
+            team_barrier(team);
+        }
+        const uint4* src4 = reinterpret_cast<const uint4*>(bm);
+        for (int w = h * 32 + lane; w < n4; w += TEAM * 32) st_stream16(row4 + w, src4[w]);
+        return;
+    }
+    int32_t sel = r.sel;
+    if (sel == -3) {
+        const int32_t hv = warp_heavy_index(p.heavy_nodes, p.n_heavy, r.node, lane);
+        sel = hv >= 0 ? hv : -2;
+    }
+    if (sel == -1 && s_root) {
+        const uint4* src4 = reinterpret_cast<const uint4*>(s_root);
+        for (int w = h * 32 + lane; w < n4; w += TEAM * 32) st_stream16(row4 + w, src4[w]);
+    } else if (sel != -2) {
+        // a prebuilt row from L2, up to eight 16-byte loads in flight per lane before the first store
+        const uint4* src4 = reinterpret_cast<const uint4*>(sel == -1 ? p.root_mask : p.heavy_masks + size_t(sel) * p.Wp);
+        int w = h * 32 + lane;
+        for (; w + 7 * TEAM * 32 < n4; w += 8 * TEAM * 32) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = ld_keep16(src4 + w + u * TEAM * 32, keep);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) st_stream16(row4 + w + u * TEAM * 32, v[u]);
+        }
+        for (; w < n4; w += TEAM * 32) st_stream16(row4 + w, ld_keep16(src4 + w, keep));
+    } else if (r.node < 0 || nc <= DESC_TOKENS) {
+        // zeros with the children's bits merged into the 16-byte stores; the children sit one per
+        // lane (a dead row has none)
+        const bool have = r.node >= 0 && lane < nc;
+        const int32_t t0 = have ? r.tk : 0;
+        // `spans` has a bit for every span that holds a child (rows of up to 32 spans; longer rows
+        // look at every span)
+        const uint32_t spans = n_it <= 32 ? __reduce_or_sync(FULL, have ? (1u << (t0 >> 12)) : 0u) : 0xffffffffu;
+        for (int it = h; it < n_it; it += TEAM) {
+            uint4 v = z;
+            if (n_it > 32 || ((spans >> it) & 1u)) {
+                uint32_t todo = __ballot_sync(FULL, have && (t0 >> 12) == it);
+                while (todo) {
+                    const int cl = __ffs(todo) - 1;
+                    todo &= todo - 1;
+                    const int32_t tc = __shfl_sync(FULL, t0, cl);
+                    if (((tc >> 7) & 31) == lane) {
+                        const uint32_t bit = 1u << (tc & 31);
+                        const int wsel = (tc >> 5) & 3;
+                        v.x |= wsel == 0 ? bit : 0u; v.y |= wsel == 1 ? bit : 0u;
+                        v.z |= wsel == 2 ? bit : 0u; v.w |= wsel == 3 ? bit : 0u;
+                    }
+                }
+            }
+            if (it * 32 + lane < n4) st_stream16(row4 + it * 32 + lane, v);
+        }
+    } else {
+        // More children than the descriptor holds and no buffer: the children are sorted by token,
+        // so the ones of a span are consecutive in the list; the warp walks the list once, 32
+        // children at a time, and its own spans that hold a child go through its patch buffer.
+        auto chunk_token = [&](int ch) -> int32_t {
+            const int j = ch * 32 + lane;
+            return j < nc ? __ldg(p.node_tok + r.cb + j) : 0x7fffffff;
+        };
+        int ch = 0;
+        int32_t t = chunk_token(0), tn = chunk_token(1);
+        for (int it = 0; it < n_it; ++it) {
+            const bool mine = (it % TEAM) == h;
+            bool dirty = false;
+            for (;;) {
+                const bool in = (t >> 12) == it;
+                if (mine && __ballot_sync(FULL, in)) {
+                    if (!dirty) {
+                        reinterpret_cast<uint4*>(patch)[lane] = z;
+                        __syncwarp();
+                        dirty = true;
+                    }
+                    if (in) atomicOr(&patch[(t >> 5) & 127], 1u << (t & 31));
+                }
+                // the chunk is used up once its last child lies in this span or before it
+                if ((__shfl_sync(FULL, t, 31) >> 12) > it) break;
+                ++ch;
+                t = tn;
+                tn = chunk_token(ch + 1);
+            }
+            if (mine) {
+                uint4 v = z;
+                if (dirty) {
+                    __syncwarp();
+                    v = reinterpret_cast<const uint4*>(patch)[lane];
+                    __syncwarp();
+                }
+                if (it * 32 + lane < n4) st_stream16(row4 + it * 32 + lane, v);
+            }
+        }
+    }
+}
+
+// dynamic shared memory of the team kernel: the root's mask row, then per team a buffer for a whole
+// mask row and one for a child list, then a patch buffer per warp
+constexpr size_t TEAM_SMEM = size_t(ROOT_SMEM_WORDS + TEAMS * (ROOT_SMEM_WORDS + DISC_HEAVY_MIN) + TEAM * TEAMS * 128) * 4;
+
+__global__ void __launch_bounds__(TEAM_THREADS, 1) disc_mask_team_kernel(const MaskParams p) {
+    extern __shared__ __align__(16) unsigned char team_smem[];
+    uint32_t* s_root_buf = reinterpret_cast<uint32_t*>(team_smem);
+    __shared__ unsigned int s_slot[TEAMS][2];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int team = warp / TEAM, h = warp % TEAM;
+    const bool fits = p.W <= ROOT_SMEM_WORDS;           // a mask row fits the buffers
+    const uint32_t* s_root = fits ? s_root_buf : nullptr;
+    uint32_t* bm = fits ? s_root_buf + ROOT_SMEM_WORDS + size_t(team) * (ROOT_SMEM_WORDS + DISC_HEAVY_MIN) : nullptr;
+    uint32_t* ts = fits ? bm + ROOT_SMEM_WORDS : nullptr;
+    uint32_t* patch = s_root_buf + ROOT_SMEM_WORDS + size_t(TEAMS) * (ROOT_SMEM_WORDS + DISC_HEAVY_MIN) + size_t(warp) * 128;
+    if (s_root) for (int w = threadIdx.x; w < p.W; w += TEAM_THREADS) s_root_buf[w] = __ldg(p.root_mask + w);
+    __syncthreads();
+    const uint64_t keep = l2_policy_evict_last();
+    const bool leader = h == 0 && lane == 0;
+    const unsigned int n = unsigned(p.n);               // n < 2^31 - 2^20, so draws past the end do not wrap
+
+    // The lane's word of a row's descriptor (read through L2: the walk kernel wrote it).
+    auto load_desc = [&](unsigned int i) -> uint32_t {
+        return i < n ? __ldcg(p.mask_out + size_t(i) * p.W + lane) : 0u;
+    };
+    // A team works three rows deep: the row in hand, the next one (its descriptor on the way), and
+    // the one after it (its index on the way back from the counter), so that neither the counter's
+    // nor L2's latency is waited for.
+    unsigned int pend = 0u;
+    if (leader) {
+        s_slot[team][0] = atomicAdd(p.work_counter, 1u);
+        s_slot[team][1] = atomicAdd(p.work_counter, 1u);
+        pend = atomicAdd(p.work_counter, 1u);
+    }
+    team_barrier(team);
+    unsigned int i_cur = s_slot[team][0], i_next = s_slot[team][1];
+    team_barrier(team);                                  // the slots are free again
+    uint32_t d_cur = load_desc(i_cur), d_next = load_desc(i_next);
+    int par = 0;
+    bool cur_prepared = false;
+    while (i_cur < n) {
+        if (leader) {
+            s_slot[team][par] = pend;
+            pend = atomicAdd(p.work_counter, 1u);
+        }
+        // After this barrier every warp of the team holds the descriptor of the row in hand (its
+        // load was issued two barriers ago), so the warp that owns the row's first span may
+        // overwrite the place it was parked in; and every warp is done with the row before, so
+        // the team's buffers are free.
+        team_barrier(team);
+        const unsigned int i_nn = s_slot[team][par];
+        par ^= 1;
+        const uint32_t d_nn = load_desc(i_nn);
+        const TeamRow rc = team_row(d_cur, lane);
+        // the next row's prebuilt mask or child list starts its way into the buffers now, if the
+        // row in hand does not need them
+        bool next_prepared = false;
+        if (bm && rc.kind == 0 && i_next < n) {
+            const TeamRow rn = team_row(d_next, lane);
+            if (rn.kind != 0) {
+                prepare_row(p, rn, bm, ts, h, lane);
+                next_prepared = true;
+            }
+        }
+        write_row_team(p, int64_t(i_cur), rc, team, h, s_root, bm, ts, cur_prepared, patch, keep, lane);
+        i_cur = i_next; d_cur = d_next; cur_prepared = next_prepared;
+        i_next = i_nn; d_next = d_nn;
+    }
+    // The last block to get here has seen every other block stop drawing: it puts the counter back
+    // to zero for the next call.
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        if (atomicAdd(p.work_counter + 1, 1u) == gridDim.x - 1) {
+            p.work_counter[0] = 0u;
+            p.work_counter[1] = 0u;
+            __threadfence();
+        }
+    }
+}
+
 // ---- host side ------------------------------------------------------------------------------------
 constexpr int MAX_DEVICES = 64;
 std::mutex g_mutex;
@@ -527,6 +859,7 @@ int resident_blocks(int* out) {
         DISC_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
         DISC_CUDA(cudaFuncSetAttribute(disc_mask_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(FUSED_SMEM)));
         DISC_CUDA(cudaFuncSetAttribute(disc_mask_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, int(FUSED_SMEM)));
+        DISC_CUDA(cudaFuncSetAttribute(disc_mask_team_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, int(TEAM_SMEM)));
         DISC_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, disc_mask_kernel<true>, FUSED_THREADS, FUSED_SMEM));
         if (per_sm > 1) per_sm = 1;          // one block per SM on purpose: few writing warps, phases aligned
         g_resident[dev] = sms * (per_sm < 1 ? 1 : per_sm);
@@ -559,6 +892,16 @@ int launch_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld, c
     const bool vec = (reinterpret_cast<uintptr_t>(mask_out) % 16 == 0) && (s->W % 4 == 0);
     int resident = 0;
     if (const int rc = resident_blocks(&resident)) return rc;
+    if (vec && s->W >= DESC_WORDS) {
+        // walks, then the rows by teams of warps, one persistent block per SM
+        disc_mask_walk_kernel<<<unsigned((n + WALK_THREADS - 1) / WALK_THREADS), WALK_THREADS, 0, st>>>(p);
+        DISC_CUDA(cudaGetLastError());
+        const int64_t want_blocks = (n + TEAMS - 1) / TEAMS;
+        const unsigned tgrid = unsigned(want_blocks < resident ? want_blocks : resident);
+        disc_mask_team_kernel<<<tgrid, TEAM_THREADS, TEAM_SMEM, st>>>(p);
+        DISC_CUDA(cudaGetLastError());
+        return DISC_OK;
+    }
     // One wave of blocks.  Every warp draws `draw` rows per round: as many as it takes to hand out
     // all rows in one round when they fit (then every block gets the same share), else 32.
     const int64_t warps = int64_t(resident) * FUSED_WARPS;

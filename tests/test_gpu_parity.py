@@ -71,7 +71,13 @@ def test_sampling_uniforms_bit_exact():
 
 @pytest.mark.parametrize("name,over,n", [("tiny", {}, 400), ("genret", {}, 3000),
                                           ("llm", dict(n_draws=200_000), 3000),
-                                          ("large", dict(n_draws=300_000), 3000)])
+                                          ("large", dict(n_draws=300_000), 3000),
+                                          # rows longer than the writer's shared-memory buffers (W = 4,100 words)
+                                          ("large", dict(n_draws=300_000, V=131_200), 2000),
+                                          # rows of 128 bytes, the shortest the two-kernel path takes
+                                          ("llm", dict(n_draws=50_000, V=1024), 2000),
+                                          # a row length that is not a multiple of 16 bytes: the one-kernel path
+                                          ("llm", dict(n_draws=100_000, V=32_003), 2000)])
 def test_mask_parity(name, over, n):
     w = scaled(name, **over)
     tok, off, G, S = _both(w)
