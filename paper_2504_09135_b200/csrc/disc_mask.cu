@@ -537,6 +537,10 @@ static_assert(TEAMS <= 15, "one named barrier per team");
 constexpr int WALK_THREADS = 256;
 
 __global__ void __launch_bounds__(WALK_THREADS) disc_mask_walk_kernel(const MaskParams p) {
+    // The team kernel is launched with programmatic stream serialisation: its blocks may be placed
+    // (and load the root's row, and draw their first rows) on SMs that this kernel's blocks have
+    // left; it reads no descriptor before this kernel has completed.
+    asm volatile("griddepcontrol.launch_dependents;");
     const int64_t i = int64_t(blockIdx.x) * WALK_THREADS + threadIdx.x;
     if (i >= p.n) return;
     const int32_t len = __ldg(p.prefix_len + i);
@@ -794,6 +798,7 @@ __global__ void __launch_bounds__(TEAM_THREADS, 1) disc_mask_team_kernel(const M
     team_barrier(team);
     unsigned int i_cur = s_slot[team][0], i_next = s_slot[team][1];
     team_barrier(team);                                  // the slots are free again
+    asm volatile("griddepcontrol.wait;" ::: "memory");   // the walks are done: their descriptors can be read
     uint32_t d_cur = load_desc(i_cur), d_next = load_desc(i_next);
     int par = 0;
     bool cur_prepared = false;
@@ -898,8 +903,13 @@ int launch_mask(const disc_set_t* s, const int32_t* prefix, int32_t prefix_ld, c
         DISC_CUDA(cudaGetLastError());
         const int64_t want_blocks = (n + TEAMS - 1) / TEAMS;
         const unsigned tgrid = unsigned(want_blocks < resident ? want_blocks : resident);
-        disc_mask_team_kernel<<<tgrid, TEAM_THREADS, TEAM_SMEM, st>>>(p);
-        DISC_CUDA(cudaGetLastError());
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(tgrid); cfg.blockDim = dim3(TEAM_THREADS); cfg.dynamicSmemBytes = TEAM_SMEM; cfg.stream = st;
+        cudaLaunchAttribute attr[1];
+        attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[0].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        DISC_CUDA(cudaLaunchKernelEx(&cfg, disc_mask_team_kernel, p));
         return DISC_OK;
     }
     // One wave of blocks.  Every warp draws `draw` rows per round: as many as it takes to hand out
