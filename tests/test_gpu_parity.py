@@ -69,6 +69,22 @@ def test_sampling_uniforms_bit_exact():
         assert np.array_equal(g.astype(np.float64), o)
 
 
+def test_mask_with_few_prefixes():
+    """Calls with fewer prefixes than the writer has teams of warps, and repeated calls (the row
+    counter must come back to zero every time)."""
+    w = scaled("llm", n_draws=50_000)
+    tok, off, G, S = _both(w)
+    prefix, plen = make_prefixes(w, tok, off, 64)
+    for n in (1, 2, 5, 6, 7, 13, 25, 64):
+        for _ in range(2):
+            g = disc.disc_mask(G, torch.as_tensor(prefix[:n], device=DEV), torch.as_tensor(plen[:n], device=DEV))
+            m, lo, hi, st = S.mask(prefix[:n], plen[:n])
+            assert np.array_equal(g["mask"].cpu().numpy().view(np.uint32), m), n
+            assert np.array_equal(g["lo"].cpu().numpy(), lo) and np.array_equal(g["hi"].cpu().numpy(), hi)
+            assert np.array_equal(g["status"].cpu().numpy(), st)
+    G.close()
+
+
 @pytest.mark.parametrize("name,over,n", [("tiny", {}, 400), ("genret", {}, 3000),
                                           ("llm", dict(n_draws=200_000), 3000),
                                           ("large", dict(n_draws=300_000), 3000),
