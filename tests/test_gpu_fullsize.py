@@ -96,6 +96,15 @@ def test_full_size_mask_stress(large):
         assert np.array_equal(lo_g[a:a + step], lo) and np.array_equal(hi_g[a:a + step], hi)
         assert np.array_equal(g["mask"][a:a + step].cpu().numpy().view(np.uint32), m)
     assert np.all(st_g == 0)
+    # The writer reads what the walks parked in the rows' own first 128 bytes just before it
+    # overwrites them, so the call is repeated over an output full of other bits: every call must
+    # give the checked result again.
+    ref = g["mask"].clone()
+    pre_d, len_d = torch.as_tensor(prefix, device=DEV), torch.as_tensor(plen, device=DEV)
+    for it in range(20):
+        g["mask"].fill_((it * 2654435761 + 12345) % 2 ** 31)
+        disc.disc_mask(G, pre_d, len_d, out=g)
+        assert torch.equal(g["mask"], ref), it
 
 
 def test_full_size_step_from_nodes_with_prebuilt_masks(large):
